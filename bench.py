@@ -1,0 +1,421 @@
+#!/usr/bin/env python
+"""Benchmark of the packed model-aggregation hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload C4]
+
+A step is one BSP iteration of every job of the workload: each block receives
+its W pushes, becomes ready in one of the rounds of the seeded arrival
+schedule, is aggregated (one packed kernel launch per round) and pulled.
+Default workload: the 12 packed concurrent jobs (661 M parameters, 31.03 GB of
+algorithmic HBM traffic per step).  Prints ONE JSON line.
+
+`value` is timed with gradients resident in HBM; `e2e` pushes from pinned host
+memory and pulls parameters back to the host inside the timed region.
+`--impl reference` times the CPU oracle on a bounded sample of the same
+workload (it is the only reference this path has).
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from workload import configs, generate  # noqa: E402
+
+METRIC = "aggregated_params_per_sec"
+UNIT = "params/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of the dominant kernel from the committed ncu capture
+# (profiles/), as measured dram bytes per algorithmic byte, keyed by the hash
+# of the kernel source it was taken from.  A changed kernel reports null.
+NCU_TRAFFIC = {"kernel_sha": None, "dram_bytes_per_algorithmic_byte": None}
+
+
+def kernel_sha() -> str:
+    h = hashlib.sha256()
+    with open(os.path.join(ROOT, "paper_2204_03211_b200", "csrc", "ps_device.cuh"), "rb") as f:
+        h.update(f.read())
+    return h.hexdigest()[:12]
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if not self.proc:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            # under load = the upper half of the samples (the sampler also sees set-up and idle gaps)
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------ our arm
+
+class Workload:
+    """The service, the device-resident gradients and the per-round call
+    arguments of one workload, prepared outside any timed region."""
+
+    def __init__(self, cfg: configs.Config, device: int, ticks: int, n_schedules: int):
+        from paper_2204_03211_b200 import binding as B
+        self.B, self.cfg, self.device = B, cfg, device
+        dev = torch.device("cuda", device)
+        arena = sum(3 * (4 * b.nelem + 256) for j in cfg.jobs for b in j.blocks) // cfg.num_contexts + (64 << 20)
+        self.svc = B.Service(device, cfg.num_contexts, arena)
+        self.slabs = []
+        for j, job in enumerate(cfg.jobs):
+            assert self.svc.register_job(**job.hparams()) == j
+            p0 = generate.init_params(cfg, j, dev)
+            for b in job.blocks:
+                self.svc.register_block(j, b.block, b.nelem, configs.initial_context(cfg, j, b.block),
+                                        p0[b.job_offset:b.job_offset + b.nelem])
+            del p0
+            self.slabs.append(generate.grad_slab(cfg, j, 0, dev))
+        torch.cuda.synchronize(dev)
+        # call arguments per schedule (= arrival pattern of one iteration) and round
+        self.schedules = []
+        for it in range(n_schedules):
+            rounds = []
+            for ready in configs.rounds_for(cfg, it, ticks):
+                jobs, blocks, workers, ptrs = [], [], [], []
+                for (j, b) in ready:
+                    job = cfg.jobs[j]
+                    blk = job.blocks[b]
+                    esz = self.slabs[j].element_size()
+                    base = self.slabs[j].data_ptr()
+                    for w in range(job.num_workers):
+                        jobs.append(j); blocks.append(b); workers.append(w)
+                        ptrs.append(base + (w * job.num_params + blk.job_offset) * esz)
+                rounds.append(dict(ready=ready, tasks=B.make_tasks(ready),
+                                   jobs=np.array(jobs, np.int32), blocks=np.array(blocks, np.int32),
+                                   workers=np.array(workers, np.int32), ptrs=np.array(ptrs, np.uint64)))
+            self.schedules.append(rounds)
+        self.params_per_step = cfg.num_params
+        self.bytes_per_step = cfg.bytes_per_round()
+
+    def step(self, k: int, stream) -> int:
+        """Push, aggregate, pull — device-resident gradients.  Returns launches."""
+        svc = self.svc
+        rounds = self.schedules[k % len(self.schedules)]
+        for r in rounds:
+            svc.push_batch(r["jobs"], r["blocks"], r["workers"], r["ptrs"])
+            svc.aggregate(r["tasks"], stream)
+            for (j, b) in r["ready"]:
+                svc.pull(j, b)
+        return len(rounds)
+
+    # ---- end to end: host gradients in, host parameters out
+
+    def prepare_host(self, pool_bytes: int):
+        total = sum(s.numel() * s.element_size() for s in self.slabs)
+        pool_bytes = min(pool_bytes, total)
+        self.pool = torch.empty(pool_bytes // 4, dtype=torch.float32).pin_memory()
+        # fill the pool with the same gradient bits (device -> host copy of the slabs' head)
+        flat = self.pool.view(torch.uint8)
+        off = 0
+        for s in self.slabs:
+            src = s.view(-1).view(torch.uint8)
+            n = min(src.numel(), flat.numel() - off)
+            if n <= 0:
+                break
+            flat[off:off + n].copy_(src[:n])
+            off += n
+        self.out = torch.empty(self.cfg.num_params, dtype=torch.float32).pin_memory()
+        self.pool_bytes = pool_bytes
+        self.h2d = total
+        self.d2h = self.cfg.num_params * 4
+
+    def step_host(self, k: int, stream) -> int:
+        svc, cfg = self.svc, self.cfg
+        rounds = self.schedules[k % len(self.schedules)]
+        pool_ptr, pool_bytes = self.pool.data_ptr(), self.pool_bytes
+        cursor = 0
+        out_ptr = self.out.data_ptr()
+        out_off = {}
+        acc = 0
+        for j, job in enumerate(cfg.jobs):
+            out_off[j] = acc
+            acc += job.num_params
+        for r in rounds:
+            for (j, b) in r["ready"]:
+                job = cfg.jobs[j]
+                nbytes = job.blocks[b].nelem * (2 if job.grad_dtype == configs.BF16 else 4)
+                for w in range(job.num_workers):
+                    if cursor + nbytes > pool_bytes:
+                        cursor = 0
+                    svc.push_host(j, b, w, pool_ptr + cursor, stream)
+                    cursor += (nbytes + 255) // 256 * 256
+            svc.aggregate(r["tasks"], stream)
+            for (j, b) in r["ready"]:
+                svc.pull_host(j, b, out_ptr + 4 * (out_off[j] + cfg.jobs[j].blocks[b].job_offset), stream)
+        return len(rounds)
+
+
+def timed(fn, steps: int, stream, dist_on: bool, device):
+    """Times `steps` calls of fn(k, stream) with CUDA events on `stream`,
+    bracketed by barrier + synchronize; returns (ms max over ranks, launches)."""
+    import torch.distributed as dist
+    torch.cuda.synchronize(device)
+    if dist_on:
+        dist.barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches = 0
+    host0 = time.perf_counter()
+    with torch.cuda.stream(stream):
+        t0.record(stream)
+        for k in range(steps):
+            launches += fn(k, stream)
+        t1.record(stream)
+    host_ms = (time.perf_counter() - host0) * 1e3
+    torch.cuda.synchronize(device)
+    if dist_on:
+        dist.barrier()
+    ms = t0.elapsed_time(t1)
+    if dist_on:
+        t = torch.tensor([ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms, launches, host_ms
+
+
+# ------------------------------------------------------------------ CPU oracle arm
+
+def oracle_sample(cfg: configs.Config, slabs=None, max_bytes: float = 9e9):
+    """Bounded sample of the workload for the CPU oracle: whole jobs, one of
+    each model where the workload has several, until the byte budget is used.
+    Returns (items for oracle.run_blocks, params, description)."""
+    from oracle import aggregator as A
+    picked, seen_models, budget = [], set(), 0
+    for j, job in enumerate(cfg.jobs):
+        cost = job.bytes_per_elem() * job.num_params
+        if job.model in seen_models or budget + cost > max_bytes:
+            continue
+        seen_models.add(job.model)
+        picked.append(j)
+        budget += cost
+    if not picked:      # a single job larger than the budget: take its first blocks
+        picked = [0]
+    items, params = [], 0
+    for j in picked:
+        job = cfg.jobs[j]
+        hp = A.HParams(**job.hparams())
+        if slabs is not None:
+            host = slabs[j].cpu()
+        else:
+            host = generate.grad_slab(cfg, j, 0)
+        host = host.view(torch.int16).numpy().view(np.uint16) if host.dtype == torch.bfloat16 else host.numpy()
+        p0 = generate.init_params(cfg, j).numpy()
+        used = 0
+        for b in job.blocks:
+            if len(picked) == 1 and used * job.bytes_per_elem() > max_bytes:
+                break
+            sl = slice(b.job_offset, b.job_offset + b.nelem)
+            p = p0[sl].copy()
+            s0 = np.zeros(b.nelem, np.float32)
+            s1 = np.zeros(b.nelem, np.float32) if job.opt == configs.ADAM else None
+            items.append((hp, 1, [host[w, sl] for w in range(job.num_workers)], p, s0, s1))
+            used += b.nelem
+        params += used
+    desc = "one aggregate of jobs %s of %s (%d blocks, %d params)" % (
+        [cfg.jobs[j].name for j in picked], cfg.name, len(items), params)
+    return items, params, desc
+
+
+def time_oracle(items, params, min_seconds: float, max_passes: int):
+    from oracle import aggregator as A
+    passes, elapsed, used = 0, 0.0, 1
+    while passes < max_passes and (elapsed < min_seconds or passes == 0):
+        t = time.perf_counter()
+        _, used = A.run_blocks(items, 0)
+        elapsed += time.perf_counter() - t
+        passes += 1
+    return params * passes / elapsed, used, passes, elapsed
+
+
+# ------------------------------------------------------------------ main
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C4", choices=sorted(configs.CONFIGS))
+    ap.add_argument("--ticks", type=int, default=16, help="rounds per iteration window of the arrival schedule")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--host-pool-gb", type=float, default=8.0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cfg = configs.CONFIGS[args.workload]()
+    config = {"workload": "%s: %d packed jobs, %d params, %d blocks, W=%s, %s arrival in <=%d rounds/step" % (
+        cfg.name, len(cfg.jobs), cfg.num_params, sum(len(j.blocks) for j in cfg.jobs),
+        sorted({j.num_workers for j in cfg.jobs}), cfg.arrival, args.ticks),
+        "l2": "inputs (%.1f GB/step) exceed L2; no flush" % (cfg.bytes_per_round() / 1e9)}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        items, params, desc = oracle_sample(cfg)
+        from oracle import aggregator as A
+        for _ in range(min(args.warmup, 1)):
+            A.run_blocks(items, 0)
+        t = time.perf_counter()
+        used = 1
+        for _ in range(args.steps):
+            _, used = A.run_blocks(items, 0)
+        dt = time.perf_counter() - t
+        val = params * args.steps / dt
+        print(json.dumps({
+            "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": config,
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": used, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}))
+        return 0
+
+    import torch.distributed as dist
+    dist_on = world > 1
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the aggregation path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if dist_on:
+        dist.init_process_group("nccl", device_id=device)
+
+    n_sched = max(1, min(args.warmup + args.steps, 8))
+    wl = Workload(cfg, local_rank, args.ticks, n_sched)
+    stream = torch.cuda.Stream(device)
+
+    for k in range(args.warmup):
+        wl.step(k, stream)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    l0 = wl.svc.launch_info()["launches"]
+    ms, launches, host_ms = timed(lambda k, s: wl.step(args.warmup + k, s), args.steps, stream, dist_on, device)
+    clocks = sampler.stop() if rank == 0 else {}
+    info = wl.svc.launch_info()
+    assert info["launches"] - l0 == launches
+    value = world * wl.params_per_step * args.steps / (ms * 1e-3)
+    achieved = wl.bytes_per_step * args.steps / (ms * 1e-3) / 1e9     # per GPU
+    peak, peak_kind = measured_peak()
+    per_launch_bytes = wl.bytes_per_step * args.steps / launches
+    sha = kernel_sha()
+    traffic = None
+    if NCU_TRAFFIC["kernel_sha"] == sha and NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"]:
+        traffic = per_launch_bytes * NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"]
+
+    e2e = None
+    if not args.no_e2e:
+        wl.prepare_host(int(args.host_pool_gb * (1 << 30)))
+        wl.step_host(0, stream)         # warm-up: allocates the staging buffers
+        torch.cuda.synchronize(device)
+        ems, _, _ = timed(wl.step_host, args.e2e_steps, stream, dist_on, device)
+        e2e = {"value": world * wl.params_per_step * args.e2e_steps / (ems * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "steps": args.e2e_steps,
+               "ms_per_step": ems / args.e2e_steps,
+               "host_pool_bytes": wl.pool_bytes}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        items, params, desc = oracle_sample(cfg, wl.slabs)
+        v, used, passes, el = time_oracle(items, params, 10.0, 50)
+        cpu = {"value": v, "unit": UNIT, "cores": used, "kind": "oracle",
+               "sample": "%s, %d passes in %.1f s" % (desc, passes, el)}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+            "hbm_gbs_algorithmic": achieved,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": traffic, "peak_source": peak_kind + " copy bandwidth",
+                         "frac_of_nominal_8TBs": achieved / 8000.0, "kernel": info["kernel"],
+                         "bytes_per_launch": per_launch_bytes, "kernel_sha": sha,
+                         "note": "duration = event time of the whole timed region / launches "
+                                 "(includes the per-launch table upload)"},
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+            "launch": {"grid": info["grid"], "block": info["block"]},
+            "host_ms_per_step": host_ms / args.steps, "clocks": clocks,
+        }
+        print(json.dumps(line))
+    wl.svc.close()
+    if dist_on:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,215 @@
+/* ps_b200.h — C ABI of the packed model-aggregation service for one B200.
+ *
+ * The service stands for the Aggregator of Parameter Service: it holds the
+ * master copy of every registered tensor block, receives the W workers'
+ * gradient shards (Push), sums them, applies the job's optimizer to the
+ * master copy in the same pass and exposes the result (Pull).  Blocks of many
+ * jobs are packed into one kernel launch.  Requests are keyed by
+ * (job ID, block ID) as in the paper's Appendix A.
+ *
+ * Conventions
+ *  - Every function returns PS_OK (0) or a negative ps_status; nothing throws
+ *    or aborts across this boundary.  On error the service is unchanged unless
+ *    the function's comment says otherwise.
+ *  - "device pointer" = address in the memory of the service's GPU.
+ *    "host pointer"   = ordinary process memory (pinned or pageable).
+ *  - `stream` arguments are a cudaStream_t passed as void* (NULL = the legacy
+ *    default stream).  Work is enqueued; functions return without waiting
+ *    unless stated.
+ *  - The service owns parameters and optimizer state; the caller owns every
+ *    gradient buffer.  The library never frees caller memory.
+ *  - A service is used from one host thread at a time (calls are serialised by
+ *    an internal mutex).
+ *
+ * Arithmetic (the paper's Section 2 says only that the server updates the
+ * master copy using the aggregated result; the optimizer equations are this
+ * library's reading).  For block b of job j at its t-th aggregate, element i:
+ *     G  = g_0[i] + g_1[i] + ... + g_{W-1}[i]      binary32, this order
+ *     G  = G * grad_scale
+ *     d  = G + wd * p[i]
+ *     SGD : v' = mom * v[i] + d;            p' = p[i] - lr * v'
+ *     ADAM: m' = b1*m[i] + (1-b1)*d;  v' = b2*v[i] + (1-b2)*d*d
+ *           p' = p[i] - (lr/(1-b1^t)) * m' / (sqrt(v')/sqrt(1-b2^t) + eps)
+ * Every operation is one IEEE-754 binary32 round-to-nearest operation with no
+ * fused multiply-add; bf16 gradients are widened exactly.  The per-block
+ * statistic is sum_i G*G in binary64.
+ */
+#ifndef PS_B200_H
+#define PS_B200_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ps_service ps_service; /* opaque */
+
+typedef enum { PS_SGD = 0, PS_ADAM = 1 } ps_opt;
+typedef enum { PS_F32 = 0, PS_BF16 = 1 } ps_dtype; /* gradient type; parameters and state are fp32 */
+
+typedef enum {
+  PS_OK = 0,
+  PS_ERR_BAD_HANDLE = -1, /* NULL or destroyed service */
+  PS_ERR_BAD_ARG = -2,    /* unknown job/block/worker/context, W < 1, nelem = 0, NULL pointer, ... */
+  PS_ERR_DUPLICATE = -3,  /* block registered twice; worker pushed twice; task listed twice */
+  PS_ERR_NOT_READY = -4,  /* a listed task has fewer than W pushes: whole call rejected */
+  PS_ERR_ALIGN = -5,      /* gradient pointer not aligned to its element size */
+  PS_ERR_NOMEM = -6,      /* context arena (or host/device allocation) exhausted */
+  PS_ERR_CUDA = -7,       /* a CUDA runtime call failed; see ps_last_cuda_error */
+  PS_ERR_NO_DEVICE = -8   /* service was created without a device (planning only) */
+} ps_status;
+
+typedef struct {
+  int opt;          /* ps_opt */
+  int grad_dtype;   /* ps_dtype */
+  int num_workers;  /* W, 1..PS_MAX_WORKERS */
+  float lr, momentum, weight_decay, beta1, beta2, eps, grad_scale;
+} ps_job_desc;
+
+typedef struct { int job, block; } ps_task;
+
+#define PS_MAX_WORKERS 256
+#define PS_DEVICE_NONE (-1)
+
+/* Options for ps_set_option / ps_get_option. */
+enum {
+  PS_OPT_CHUNK_ELEMS = 1,  /* elements per (job,block,chunk) descriptor; 0 = automatic.
+                              Must be a multiple of 1024 (<= 2^20) when non-zero. */
+  PS_OPT_CTAS_PER_SM = 2,  /* persistent CTAs per SM; 0 = automatic */
+  PS_OPT_SORT_TASKS = 3,   /* 1 (default): heaviest chunks first inside a launch; 0: caller's order */
+  PS_OPT_KERNEL = 4        /* kernel variant: 0 = automatic; see ps_kernel_name */
+};
+
+/* Creates an Aggregator service on GPU `device` with `num_contexts` contexts
+ * (paper Section 3.1: an Aggregator holds the master copies of the tensors
+ * assigned to it; here a context is one arena of `arena_bytes_per_ctx` bytes of
+ * device memory that holds parameters and optimizer state).  Allocates the
+ * arenas with cudaMalloc.  device = PS_DEVICE_NONE builds a planning-only
+ * service: registration, push bookkeeping and ps_plan work, no device memory
+ * exists and ps_aggregate/ps_pull/ps_migrate_block return PS_ERR_NO_DEVICE.
+ * Errors: BAD_ARG (out NULL, num_contexts < 1), NOMEM, CUDA. */
+int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes_per_ctx);
+
+/* Frees the arenas and all service-owned memory after synchronising the
+ * device work the service enqueued.  Pointers from ps_pull become invalid. */
+int ps_destroy(ps_service* svc);
+
+/* Registers a training job (paper Section 4: Agents register the job with the
+ * manager; Appendix A: the job ID travels with every request).  `desc` is a
+ * host pointer, copied.  *job_out receives the job ID (0, 1, 2, ...).
+ * Errors: BAD_ARG (opt/dtype unknown, W out of range, NULL). */
+int ps_register_job(ps_service* svc, const ps_job_desc* desc, int* job_out);
+
+/* Registers block `block` (>= 0, caller-chosen, unique within the job) of
+ * `nelem` fp32 parameters in context `ctx` — the per-tensor Init of the
+ * paper's Appendix A.  `init_params_or_null` may be a host or a device pointer
+ * to nelem floats (copied before return) or NULL (zeros).  Optimizer state
+ * starts at zero and the step counter at 0.  Synchronous.
+ * Errors: BAD_ARG, DUPLICATE, NOMEM, CUDA. */
+int ps_register_block(ps_service* svc, int job, int block, size_t nelem, int ctx,
+                      const float* init_params_or_null);
+
+/* Push (paper Section 4, Appendix A): records worker `worker`'s gradient shard
+ * for (job, block).  Zero-copy: `grad_dev_ptr` is a device pointer to nelem
+ * contiguous values of the job's grad_dtype; it must stay valid and unmodified
+ * until the ps_aggregate that consumes it has completed on its stream.  The
+ * task is ready once all W workers have pushed.  16-byte aligned pointers take
+ * the vector path, others a scalar path with identical results.
+ * Errors: BAD_ARG, DUPLICATE (this worker already pushed this iteration; the
+ * paper has one request per task per iteration), ALIGN. */
+int ps_push(ps_service* svc, int job, int block, int worker, const void* grad_dev_ptr);
+
+/* n pushes in one call (host arrays of length n).  All-or-nothing. */
+int ps_push_batch(ps_service* svc, int n, const int* jobs, const int* blocks, const int* workers,
+                  const void* const* grad_dev_ptrs);
+
+/* Push from host memory: copies nelem gradient values from `grad_host_ptr`
+ * into a service-owned device staging buffer (allocated on first use for this
+ * block) with cudaMemcpyAsync on `stream`, then records the push.  The host
+ * buffer must stay valid until that copy completes; the ps_aggregate that
+ * consumes the push must be enqueued on the same stream (or one ordered after
+ * it).  Errors as ps_push, plus NOMEM, CUDA, NO_DEVICE. */
+int ps_push_host(ps_service* svc, int job, int block, int worker, const void* grad_host_ptr,
+                 void* stream);
+
+/* Aggregates every task in `ready` (host array, any mix of jobs) in ONE kernel
+ * launch on `stream`: sum of the W shards in worker order, optimizer update of
+ * the master copy and state, per-block squared gradient norm (the paper's
+ * Section 3.3 packs many jobs' aggregation tasks onto a shared Aggregator;
+ * Figure 1: update after all workers pushed).  On success each listed block's
+ * pushes are consumed and its step counter is incremented.  n_ready = 0 is a
+ * no-op.  If a listed block is under migration the launch is ordered after the
+ * copy (Appendix B, "Data Consistency").
+ * Errors (nothing launched, nothing changed): BAD_ARG, DUPLICATE, NOT_READY,
+ * NO_DEVICE, NOMEM, CUDA. */
+int ps_aggregate(ps_service* svc, const ps_task* ready, int n_ready, void* stream);
+
+/* Pull (paper Section 4): *params_dev_ptr_out receives a device pointer to the
+ * block's nelem fp32 parameters.  Borrowed; stable until the block is migrated
+ * or the service destroyed; contents are defined once the last ps_aggregate /
+ * ps_migrate_block enqueued for the block has completed on its stream. */
+int ps_pull(ps_service* svc, int job, int block, const float** params_dev_ptr_out);
+
+/* Pull into host memory: enqueues a device-to-host copy of the parameters on
+ * `stream` (ordered after the block's last aggregate/migration). */
+int ps_pull_host(ps_service* svc, int job, int block, float* params_host_dst, void* stream);
+
+/* Moves the block's master copy — parameters, optimizer state and step
+ * counter — to context `dst_ctx` (paper Section 3.2 and Appendix B: the old
+ * Aggregator copies the tensor's contents to the new one, which must not
+ * update it before the copy has landed).  The copy is enqueued on `stream`
+ * after the block's last aggregate; later aggregates of the block wait for it;
+ * the source memory is released when the copy has completed.  Pending pushes
+ * stay with the block.  dst_ctx equal to the current context is a no-op.
+ * Errors: BAD_ARG, NOMEM (block stays where it was), NO_DEVICE, CUDA. */
+int ps_migrate_block(ps_service* svc, int job, int block, int dst_ctx, void* stream);
+
+/* Per-block statistics of the last aggregate (paper Section 3.1: profilers feed
+ * the manager): squared norm of the aggregated gradient and the step counter.
+ * Waits for the block's last aggregate to finish.  Either out pointer may be
+ * NULL.  Before the first aggregate the norm is 0 and the step 0. */
+int ps_block_stats(ps_service* svc, int job, int block, double* grad_sqnorm_out,
+                   unsigned long long* step_out);
+
+/* Device pointers to the block's optimizer state (momentum | Adam m, and
+ * Adam v or NULL) and its current context; for tests and checkpoints. */
+int ps_block_state(ps_service* svc, int job, int block, const float** state0_dev_ptr_out,
+                   const float** state1_dev_ptr_out, int* ctx_out);
+
+/* One (job, block, chunk) descriptor as the kernel will see it. */
+typedef struct {
+  int job, block;
+  unsigned long long elem_begin, elem_count;
+  int num_workers;
+  int vector_path; /* 1 if every pointer of the task allows 128-bit accesses */
+} ps_chunk_info;
+
+/* Builds the packed task table for `ready` exactly as ps_aggregate would,
+ * without launching or consuming anything, and writes up to `cap` chunk
+ * descriptors (in the order CTAs will claim them) to `out` (host, may be NULL);
+ * *n_chunks_out receives the total.  Works on planning-only services.
+ * Errors as ps_aggregate's validation. */
+int ps_plan(ps_service* svc, const ps_task* ready, int n_ready, ps_chunk_info* out, size_t cap,
+            size_t* n_chunks_out);
+
+int ps_set_option(ps_service* svc, int option, long long value);
+int ps_get_option(ps_service* svc, int option, long long* value_out);
+
+/* Bytes in use / largest free range of a context's arena. */
+int ps_arena_info(ps_service* svc, int ctx, size_t* used_out, size_t* largest_free_out);
+
+/* Number of aggregation kernels launched so far and the grid/block size and
+ * variant name of the last one (for launch accounting in benchmarks). */
+int ps_launch_info(ps_service* svc, unsigned long long* launches_out, int* grid_out, int* block_out,
+                   const char** kernel_name_out);
+
+const char* ps_strerror(int status);
+/* Text of the last CUDA error seen by this service ("" if none). */
+const char* ps_last_cuda_error(ps_service* svc);
+const char* ps_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PS_B200_H */

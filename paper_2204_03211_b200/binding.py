@@ -1,0 +1,286 @@
+"""ctypes binding of the C-ABI library (include/ps_b200.h).
+
+Argument marshalling only: every step of the aggregation path runs in the
+library's CUDA kernels.  The module-level functions carry the names of the C
+entry points; `Service` is a thin object wrapper over the same calls.  If the
+shared library is missing or cannot be loaded the import of `load()` raises —
+there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libps_b200.so")
+
+PS_SGD, PS_ADAM = 0, 1
+PS_F32, PS_BF16 = 0, 1
+PS_OK = 0
+PS_ERR_BAD_HANDLE, PS_ERR_BAD_ARG, PS_ERR_DUPLICATE, PS_ERR_NOT_READY = -1, -2, -3, -4
+PS_ERR_ALIGN, PS_ERR_NOMEM, PS_ERR_CUDA, PS_ERR_NO_DEVICE = -5, -6, -7, -8
+PS_DEVICE_NONE = -1
+PS_MAX_WORKERS = 256
+PS_OPT_CHUNK_ELEMS, PS_OPT_CTAS_PER_SM, PS_OPT_SORT_TASKS, PS_OPT_KERNEL = 1, 2, 3, 4
+
+
+class ps_job_desc(C.Structure):
+    _fields_ = [("opt", C.c_int), ("grad_dtype", C.c_int), ("num_workers", C.c_int),
+                ("lr", C.c_float), ("momentum", C.c_float), ("weight_decay", C.c_float),
+                ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float), ("grad_scale", C.c_float)]
+
+
+class ps_task(C.Structure):
+    _fields_ = [("job", C.c_int), ("block", C.c_int)]
+
+
+class ps_chunk_info(C.Structure):
+    _fields_ = [("job", C.c_int), ("block", C.c_int), ("elem_begin", C.c_ulonglong),
+                ("elem_count", C.c_ulonglong), ("num_workers", C.c_int), ("vector_path", C.c_int)]
+
+
+class PsError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        msg = "%s: %s (%d)" % (where, ps_strerror(status), status)
+        super().__init__(msg + (": " + detail if detail else ""))
+
+
+_lib = None
+
+_SIGNATURES = {
+    "ps_create": (C.c_int, [C.POINTER(C.c_void_p), C.c_int, C.c_int, C.c_size_t]),
+    "ps_destroy": (C.c_int, [C.c_void_p]),
+    "ps_register_job": (C.c_int, [C.c_void_p, C.POINTER(ps_job_desc), C.POINTER(C.c_int)]),
+    "ps_register_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_size_t, C.c_int, C.c_void_p]),
+    "ps_push": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]),
+    "ps_push_batch": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ps_push_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
+    "ps_aggregate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
+    "ps_pull": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p)]),
+    "ps_pull_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
+    "ps_migrate_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]),
+    "ps_block_stats": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_ulonglong)]),
+    "ps_block_state": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p),
+                                 C.POINTER(C.c_int)]),
+    "ps_plan": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]),
+    "ps_set_option": (C.c_int, [C.c_void_p, C.c_int, C.c_longlong]),
+    "ps_get_option": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_longlong)]),
+    "ps_arena_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "ps_launch_info": (C.c_int, [C.c_void_p, C.POINTER(C.c_ulonglong), C.POINTER(C.c_int), C.POINTER(C.c_int),
+                                 C.POINTER(C.c_char_p)]),
+    "ps_strerror": (C.c_char_p, [C.c_int]),
+    "ps_last_cuda_error": (C.c_char_p, [C.c_void_p]),
+    "ps_version": (C.c_char_p, []),
+}
+
+
+def load():
+    """Loads libps_b200.so (built in-tree by paper_2204_03211_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("%s is missing: run `python -m paper_2204_03211_b200.build` "
+                              "(there is no fallback path)" % LIB_PATH)
+        lib = C.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def ps_strerror(status: int) -> str:
+    return load().ps_strerror(status).decode()
+
+
+def ps_version() -> str:
+    return load().ps_version().decode()
+
+
+def _check(rc: int, where: str, svc=None):
+    if rc != PS_OK:
+        detail = load().ps_last_cuda_error(svc).decode() if (svc and rc == PS_ERR_CUDA) else ""
+        raise PsError(rc, where, detail)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        return 0
+    return int(getattr(stream, "cuda_stream", stream))
+
+
+def _ptr(x) -> int:
+    """Address of a torch tensor / numpy array / raw integer."""
+    if x is None:
+        return 0
+    if hasattr(x, "data_ptr"):
+        return int(x.data_ptr())
+    if hasattr(x, "ctypes"):
+        return int(x.ctypes.data)
+    return int(x)
+
+
+# ---- module-level functions with the C names --------------------------------
+
+def ps_create(device: int, num_contexts: int, arena_bytes_per_ctx: int) -> int:
+    h = C.c_void_p()
+    _check(load().ps_create(C.byref(h), device, num_contexts, arena_bytes_per_ctx), "ps_create")
+    return h.value
+
+
+def ps_destroy(svc):
+    _check(load().ps_destroy(svc), "ps_destroy")
+
+
+def ps_register_job(svc, opt=PS_SGD, grad_dtype=PS_F32, num_workers=1, lr=0.1, momentum=0.0, weight_decay=0.0,
+                    beta1=0.9, beta2=0.999, eps=1e-8, grad_scale=1.0) -> int:
+    d = ps_job_desc(opt, grad_dtype, num_workers, lr, momentum, weight_decay, beta1, beta2, eps, grad_scale)
+    job = C.c_int(-1)
+    _check(load().ps_register_job(svc, C.byref(d), C.byref(job)), "ps_register_job", svc)
+    return job.value
+
+
+def ps_register_block(svc, job: int, block: int, nelem: int, ctx: int = 0, init_params=None):
+    _check(load().ps_register_block(svc, job, block, nelem, ctx, _ptr(init_params)), "ps_register_block", svc)
+
+
+def ps_push(svc, job: int, block: int, worker: int, grad):
+    _check(load().ps_push(svc, job, block, worker, _ptr(grad)), "ps_push", svc)
+
+
+def ps_push_batch(svc, jobs, blocks, workers, ptrs):
+    """jobs/blocks/workers: contiguous int32 numpy arrays; ptrs: uint64 numpy array."""
+    n = len(jobs)
+    _check(load().ps_push_batch(svc, n, jobs.ctypes.data, blocks.ctypes.data, workers.ctypes.data,
+                                ptrs.ctypes.data), "ps_push_batch", svc)
+
+
+def ps_push_host(svc, job: int, block: int, worker: int, grad_host, stream=None):
+    _check(load().ps_push_host(svc, job, block, worker, _ptr(grad_host), _stream_ptr(stream)), "ps_push_host", svc)
+
+
+def make_tasks(pairs):
+    """[(job, block), ...] -> ctypes array of ps_task (reusable across calls)."""
+    arr = (ps_task * len(pairs))()
+    for i, (j, b) in enumerate(pairs):
+        arr[i].job, arr[i].block = j, b
+    return arr
+
+
+def ps_aggregate(svc, ready, stream=None):
+    tasks = ready if isinstance(ready, C.Array) else make_tasks(list(ready))
+    _check(load().ps_aggregate(svc, tasks, len(tasks), _stream_ptr(stream)), "ps_aggregate", svc)
+
+
+def ps_pull(svc, job: int, block: int) -> int:
+    out = C.c_void_p()
+    _check(load().ps_pull(svc, job, block, C.byref(out)), "ps_pull", svc)
+    return out.value
+
+
+def ps_pull_host(svc, job: int, block: int, dst_host, stream=None):
+    _check(load().ps_pull_host(svc, job, block, _ptr(dst_host), _stream_ptr(stream)), "ps_pull_host", svc)
+
+
+def ps_migrate_block(svc, job: int, block: int, dst_ctx: int, stream=None):
+    _check(load().ps_migrate_block(svc, job, block, dst_ctx, _stream_ptr(stream)), "ps_migrate_block", svc)
+
+
+def ps_block_stats(svc, job: int, block: int):
+    sq, step = C.c_double(), C.c_ulonglong()
+    _check(load().ps_block_stats(svc, job, block, C.byref(sq), C.byref(step)), "ps_block_stats", svc)
+    return sq.value, step.value
+
+
+def ps_block_state(svc, job: int, block: int):
+    s0, s1, ctx = C.c_void_p(), C.c_void_p(), C.c_int()
+    _check(load().ps_block_state(svc, job, block, C.byref(s0), C.byref(s1), C.byref(ctx)), "ps_block_state", svc)
+    return s0.value, s1.value, ctx.value
+
+
+def ps_plan(svc, ready):
+    tasks = ready if isinstance(ready, C.Array) else make_tasks(list(ready))
+    n = C.c_size_t()
+    _check(load().ps_plan(svc, tasks, len(tasks), None, 0, C.byref(n)), "ps_plan", svc)
+    out = (ps_chunk_info * max(1, n.value))()
+    _check(load().ps_plan(svc, tasks, len(tasks), out, n.value, C.byref(n)), "ps_plan", svc)
+    return [out[i] for i in range(n.value)]
+
+
+def ps_set_option(svc, option: int, value: int):
+    _check(load().ps_set_option(svc, option, value), "ps_set_option", svc)
+
+
+def ps_get_option(svc, option: int) -> int:
+    v = C.c_longlong()
+    _check(load().ps_get_option(svc, option, C.byref(v)), "ps_get_option", svc)
+    return v.value
+
+
+def ps_arena_info(svc, ctx: int):
+    used, free = C.c_size_t(), C.c_size_t()
+    _check(load().ps_arena_info(svc, ctx, C.byref(used), C.byref(free)), "ps_arena_info", svc)
+    return used.value, free.value
+
+
+def ps_launch_info(svc):
+    n, g, b, name = C.c_ulonglong(), C.c_int(), C.c_int(), C.c_char_p()
+    _check(load().ps_launch_info(svc, C.byref(n), C.byref(g), C.byref(b), C.byref(name)), "ps_launch_info", svc)
+    return dict(launches=n.value, grid=g.value, block=b.value, kernel=(name.value or b"").decode())
+
+
+# ---- object wrapper -----------------------------------------------------------
+
+class Service:
+    """Owns one ps_service handle; methods are the C entry points without the
+    `ps_` prefix and the handle argument."""
+
+    def __init__(self, device: int = 0, num_contexts: int = 1, arena_bytes_per_ctx: int = 1 << 30):
+        self.handle = ps_create(device, num_contexts, arena_bytes_per_ctx)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            ps_destroy(self.handle)
+            self.handle = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def view(self, ptr: int, nelem: int, device: int | None = None):
+        """fp32 torch view of `nelem` elements of service-owned device memory
+        (for reading results in tests; no copy)."""
+        import torch
+
+        class _Mem:
+            pass
+
+        m = _Mem()
+        m.__cuda_array_interface__ = {"shape": (nelem,), "typestr": "<f4", "data": (ptr, False), "version": 2}
+        return torch.as_tensor(m, device="cuda" if device is None else "cuda:%d" % device)
+
+
+def _bind(name):
+    fn = globals()["ps_" + name]
+
+    def method(self, *a, **k):
+        return fn(self.handle, *a, **k)
+
+    method.__name__ = name
+    method.__doc__ = fn.__doc__
+    return method
+
+
+for _n in ("register_job", "register_block", "push", "push_batch", "push_host", "aggregate", "pull", "pull_host",
+           "migrate_block", "block_stats", "block_state", "plan", "set_option", "get_option", "arena_info",
+           "launch_info"):
+    setattr(Service, _n, _bind(_n))

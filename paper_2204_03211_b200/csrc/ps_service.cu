@@ -1,0 +1,799 @@
+// Host runtime and C ABI of the packed model-aggregation service
+// (declarations and contracts: include/ps_b200.h).
+//
+// Host side = the Aggregator's bookkeeping: registry of jobs and blocks keyed
+// by (job ID, block ID) (paper Appendix A), push counting per iteration (BSP,
+// paper Figure 1), the block -> context map that stands for the Agents'
+// mapping table (paper Section 3.1), migration with the not-before-the-copy
+// rule (paper Appendix B), and the builder of the packed task table that one
+// kernel launch consumes (paper Section 3.3: tasks of many jobs share one
+// Aggregator).  Every arithmetic step runs in the kernels of ps_device.cuh;
+// there is no host fallback.
+#include "../../include/ps_b200.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "arena.h"
+#include "ps_device.cuh"
+
+namespace psb {
+
+constexpr uint32_t kMagic = 0x50534232u;   // "PSB2"
+constexpr int kSlots = 4;                  // task tables in flight
+constexpr unsigned int kMaxChunk = 1u << 20;
+
+struct Job {
+  ps_job_desc d;
+  std::vector<int> block_of_id;            // block id -> index into Service::blocks, -1 = none
+  size_t grad_esize() const { return d.grad_dtype == PS_BF16 ? 2 : 4; }
+  int nstate() const { return d.opt == PS_ADAM ? 2 : 1; }
+};
+
+struct Block {
+  int job = 0, id = 0;
+  size_t nelem = 0;
+  int ctx = 0;
+  size_t off = 0, bytes = 0;               // one arena range: p | s0 | s1
+  size_t sec = 0;                          // byte stride between p, s0, s1
+  unsigned long long step = 0;
+  std::vector<const void*> pushed;         // W entries, nullptr = not pushed
+  int npushed = 0;
+  unsigned int stat_idx = 0;
+  unsigned long long mark = 0;             // duplicate detection inside one ready list
+  int last_slot = -1;                      // slot of the last aggregate
+  unsigned long long last_slot_gen = 0;
+  cudaEvent_t mig_event = nullptr;
+  bool mig_pending = false;
+  void* staging = nullptr;                 // device buffer for ps_push_host
+  size_t staging_row = 0;
+};
+
+struct Ctx {
+  char* base = nullptr;
+  Arena arena;
+};
+
+struct PendingFree {
+  int ctx;
+  size_t off, bytes;
+  cudaEvent_t ev;                          // owned by the block; only queried here
+  int block;
+};
+
+struct Slot {
+  unsigned char* host = nullptr;           // pinned
+  unsigned char* dev = nullptr;
+  size_t cap = 0;
+  double* partials = nullptr;
+  size_t partial_cap = 0;
+  cudaEvent_t done = nullptr;
+  bool inflight = false;
+  unsigned long long gen = 0;
+};
+
+struct Plan {                              // one built task table (host copy)
+  std::vector<unsigned char> bytes;
+  std::vector<int> order;                  // block indices in table order
+  unsigned int total_chunks = 0, chunk_elems = 0;
+};
+
+}  // namespace psb
+
+using namespace psb;
+
+struct ps_service {
+  uint32_t magic = kMagic;
+  int device = PS_DEVICE_NONE;
+  int num_sms = 148;
+  std::mutex mu;
+  std::vector<Ctx> ctxs;
+  std::vector<Job> jobs;
+  std::vector<Block> blocks;
+  std::vector<PendingFree> pending_free;
+  PsJobDev* jobs_dev = nullptr;
+  size_t jobs_dev_cap = 0;
+  PsStat* stats_dev = nullptr;
+  size_t stats_dev_cap = 0;
+  Slot slots[kSlots];
+  int next_slot = 0;
+  unsigned long long gen = 0;              // ready-list generation
+  long long opt_chunk = 0, opt_ctas = 0, opt_sort = 1, opt_kernel = 0;
+  int occ_ctas = 0;
+  unsigned long long launches = 0;
+  int last_grid = 0, last_block = 0;
+  const char* last_kernel = "none";
+  std::string cuda_err;
+};
+
+namespace {
+
+#define PS_CUDA(svc, call)                                                            \
+  do {                                                                                \
+    cudaError_t e__ = (call);                                                         \
+    if (e__ != cudaSuccess) {                                                         \
+      (svc)->cuda_err = std::string(#call) + ": " + cudaGetErrorString(e__);          \
+      return PS_ERR_CUDA;                                                             \
+    }                                                                                 \
+  } while (0)
+
+bool alive(const ps_service* s) { return s && s->magic == kMagic; }
+bool has_device(const ps_service* s) { return s->device >= 0; }
+
+int find_block(ps_service* s, int job, int block) {
+  if (job < 0 || job >= (int)s->jobs.size() || block < 0) return -1;
+  const Job& j = s->jobs[job];
+  if (block >= (int)j.block_of_id.size()) return -1;
+  return j.block_of_id[block];
+}
+
+float* blk_p(ps_service* s, const Block& b) { return reinterpret_cast<float*>(s->ctxs[b.ctx].base + b.off); }
+float* blk_s0(ps_service* s, const Block& b) { return reinterpret_cast<float*>(s->ctxs[b.ctx].base + b.off + b.sec); }
+float* blk_s1(ps_service* s, const Block& b) {
+  return s->jobs[b.job].nstate() == 2 ? reinterpret_cast<float*>(s->ctxs[b.ctx].base + b.off + 2 * b.sec) : nullptr;
+}
+
+// Releases source ranges of finished migrations.  With wait = true blocks
+// until every pending copy has completed.
+int reap_frees(ps_service* s, bool wait) {
+  size_t keep = 0;
+  for (size_t i = 0; i < s->pending_free.size(); ++i) {
+    PendingFree& f = s->pending_free[i];
+    cudaError_t q = wait ? cudaEventSynchronize(f.ev) : cudaEventQuery(f.ev);
+    if (q == cudaSuccess) {
+      s->ctxs[f.ctx].arena.release(f.off, f.bytes);
+    } else if (q == cudaErrorNotReady) {
+      s->pending_free[keep++] = f;
+    } else {
+      s->cuda_err = std::string("migration event: ") + cudaGetErrorString(q);
+      return PS_ERR_CUDA;
+    }
+  }
+  s->pending_free.resize(keep);
+  return PS_OK;
+}
+
+int arena_alloc(ps_service* s, int ctx, size_t bytes, size_t* off_out) {
+  if (has_device(s)) {
+    int rc = reap_frees(s, false);
+    if (rc) return rc;
+  }
+  size_t off = s->ctxs[ctx].arena.alloc(bytes);
+  if (off == Arena::kNone && has_device(s) && !s->pending_free.empty()) {
+    int rc = reap_frees(s, true);
+    if (rc) return rc;
+    off = s->ctxs[ctx].arena.alloc(bytes);
+  }
+  if (off == Arena::kNone) return PS_ERR_NOMEM;
+  *off_out = off;
+  return PS_OK;
+}
+
+template <typename T>
+int grow_dev(ps_service* s, T** buf, size_t* cap, size_t need, bool zero_new) {
+  if (need <= *cap) return PS_OK;
+  size_t ncap = *cap ? *cap : 64;
+  while (ncap < need) ncap *= 2;
+  T* nbuf = nullptr;
+  PS_CUDA(s, cudaMalloc(&nbuf, ncap * sizeof(T)));
+  PS_CUDA(s, cudaDeviceSynchronize());
+  if (zero_new) PS_CUDA(s, cudaMemset(nbuf, 0, ncap * sizeof(T)));
+  if (*buf) {
+    PS_CUDA(s, cudaMemcpy(nbuf, *buf, *cap * sizeof(T), cudaMemcpyDeviceToDevice));
+    PS_CUDA(s, cudaFree(*buf));
+  }
+  *buf = nbuf;
+  *cap = ncap;
+  return PS_OK;
+}
+
+// Validates a ready list (no state change besides the duplicate marks) and
+// returns the block indices in list order.
+int validate_ready(ps_service* s, const ps_task* ready, int n_ready, std::vector<int>* out) {
+  if (n_ready < 0 || (n_ready > 0 && !ready)) return PS_ERR_BAD_ARG;
+  const unsigned long long gen = ++s->gen;
+  out->clear();
+  out->reserve(n_ready);
+  for (int i = 0; i < n_ready; ++i) {
+    const int bi = find_block(s, ready[i].job, ready[i].block);
+    if (bi < 0) return PS_ERR_BAD_ARG;
+    Block& b = s->blocks[bi];
+    if (b.mark == gen) return PS_ERR_DUPLICATE;
+    b.mark = gen;
+    out->push_back(bi);
+  }
+  for (int bi : *out) {
+    const Block& b = s->blocks[bi];
+    if (b.npushed != s->jobs[b.job].d.num_workers) return PS_ERR_NOT_READY;
+  }
+  return PS_OK;
+}
+
+size_t bytes_per_elem(const Job& j) { return (size_t)j.d.num_workers * j.grad_esize() + 8 * (1 + j.nstate()); }
+
+unsigned int pick_chunk_elems(ps_service* s, const std::vector<int>& idx, int grid_cap) {
+  if (s->opt_chunk > 0) return (unsigned int)s->opt_chunk;
+  // Aim for ~16 chunks per resident CTA so that the tail of a launch is short,
+  // within [1024, 4096] elements.
+  unsigned long long total = 0;
+  for (int bi : idx) total += s->blocks[bi].nelem;
+  unsigned long long want = total / ((unsigned long long)grid_cap * 16ull);
+  unsigned int c = 4096;
+  while (c > 1024 && c > want) c >>= 1;
+  return c;
+}
+
+int grid_cap(ps_service* s) {
+  const int per_sm = s->opt_ctas > 0 ? (int)s->opt_ctas : (s->occ_ctas > 0 ? s->occ_ctas : 3);
+  return s->num_sms * per_sm;
+}
+
+// Builds the task table for the validated blocks `idx`.
+int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
+  const size_t n = idx.size();
+  plan->order = idx;
+  plan->chunk_elems = pick_chunk_elems(s, idx, grid_cap(s));
+  const unsigned int ce = plan->chunk_elems;
+  if (s->opt_sort) {
+    // heaviest chunks first: the launch's tail is then made of light chunks
+    std::stable_sort(plan->order.begin(), plan->order.end(), [&](int a, int b) {
+      const Block& A = s->blocks[a];
+      const Block& B = s->blocks[b];
+      const size_t ca = std::min<size_t>(A.nelem, ce) * bytes_per_elem(s->jobs[A.job]);
+      const size_t cb = std::min<size_t>(B.nelem, ce) * bytes_per_elem(s->jobs[B.job]);
+      return ca > cb;
+    });
+  }
+  size_t nptr = 0;
+  for (int bi : plan->order) nptr += s->jobs[s->blocks[bi].job].d.num_workers;
+  const size_t tasks_off = sizeof(PsTableHdr);
+  const size_t starts_off = tasks_off + n * sizeof(PsTaskDev);
+  const size_t ptrs_off = (starts_off + n * sizeof(unsigned int) + 15) / 16 * 16;
+  plan->bytes.assign(ptrs_off + nptr * sizeof(void*), 0);
+  unsigned char* base = plan->bytes.data();
+  PsTaskDev* tasks = reinterpret_cast<PsTaskDev*>(base + tasks_off);
+  unsigned int* starts = reinterpret_cast<unsigned int*>(base + starts_off);
+  const void** ptrs = reinterpret_cast<const void**>(base + ptrs_off);
+  unsigned long long chunk = 0;
+  size_t row = 0;
+  for (size_t i = 0; i < n; ++i) {
+    const Block& b = s->blocks[plan->order[i]];
+    const Job& j = s->jobs[b.job];
+    PsTaskDev& t = tasks[i];
+    t.p = blk_p(s, b);
+    t.s0 = blk_s0(s, b);
+    t.s1 = blk_s1(s, b);
+    t.nelem = b.nelem;
+    t.shard_row = (unsigned int)row;
+    t.first_chunk = (unsigned int)chunk;
+    t.nchunks = (unsigned int)((b.nelem + ce - 1) / ce);
+    t.ticket = 0;
+    const unsigned long long step = b.step + 1;
+    t.ss_t = (float)((double)j.d.lr / (1.0 - std::pow((double)j.d.beta1, (double)step)));
+    t.sbc2_t = (float)std::sqrt(1.0 - std::pow((double)j.d.beta2, (double)step));
+    t.job = b.job;
+    t.stat_idx = b.stat_idx;
+    t.step = step;
+    unsigned int vec = 1;
+    for (int w = 0; w < j.d.num_workers; ++w) {
+      ptrs[row + w] = b.pushed[w];
+      if (reinterpret_cast<uintptr_t>(b.pushed[w]) & 15u) vec = 0;
+    }
+    t.vec_ok = vec;
+    starts[i] = t.first_chunk;
+    row += j.d.num_workers;
+    chunk += t.nchunks;
+    if (chunk > 0xfffffff0ull) return PS_ERR_BAD_ARG;
+  }
+  plan->total_chunks = (unsigned int)chunk;
+  PsTableHdr* h = reinterpret_cast<PsTableHdr*>(base);
+  h->counter = 0;
+  h->n_tasks = (unsigned int)n;
+  h->total_chunks = plan->total_chunks;
+  h->chunk_elems = ce;
+  h->tasks_off = (unsigned int)tasks_off;
+  h->starts_off = (unsigned int)starts_off;
+  h->ptrs_off = (unsigned int)ptrs_off;
+  return PS_OK;
+}
+
+int acquire_slot(ps_service* s, size_t table_bytes, size_t nchunks, Slot** out) {
+  Slot& sl = s->slots[s->next_slot];
+  if (sl.inflight) {
+    PS_CUDA(s, cudaEventSynchronize(sl.done));
+    sl.inflight = false;
+  }
+  if (!sl.done) PS_CUDA(s, cudaEventCreateWithFlags(&sl.done, cudaEventDisableTiming));
+  if (table_bytes > sl.cap) {
+    size_t ncap = std::max<size_t>(table_bytes * 2, 1 << 16);
+    if (sl.host) PS_CUDA(s, cudaFreeHost(sl.host));
+    if (sl.dev) PS_CUDA(s, cudaFree(sl.dev));
+    sl.host = nullptr; sl.dev = nullptr; sl.cap = 0;
+    PS_CUDA(s, cudaHostAlloc(&sl.host, ncap, cudaHostAllocDefault));
+    PS_CUDA(s, cudaMalloc(&sl.dev, ncap));
+    sl.cap = ncap;
+  }
+  if (nchunks > sl.partial_cap) {
+    size_t ncap = std::max<size_t>(nchunks * 2, 1 << 12);
+    if (sl.partials) PS_CUDA(s, cudaFree(sl.partials));
+    sl.partials = nullptr; sl.partial_cap = 0;
+    PS_CUDA(s, cudaMalloc(&sl.partials, ncap * sizeof(double)));
+    sl.partial_cap = ncap;
+  }
+  sl.gen = s->gen;
+  *out = &sl;
+  return PS_OK;
+}
+
+// Makes `stream` wait for everything enqueued so far that touches block b.
+int order_after_block(ps_service* s, Block& b, cudaStream_t stream) {
+  if (b.last_slot >= 0) {
+    Slot& sl = s->slots[b.last_slot];
+    if (sl.inflight && sl.gen == b.last_slot_gen) PS_CUDA(s, cudaStreamWaitEvent(stream, sl.done, 0));
+  }
+  if (b.mig_pending) {
+    cudaError_t q = cudaEventQuery(b.mig_event);
+    if (q == cudaSuccess) b.mig_pending = false;
+    else if (q == cudaErrorNotReady) PS_CUDA(s, cudaStreamWaitEvent(stream, b.mig_event, 0));
+    else { s->cuda_err = cudaGetErrorString(q); return PS_ERR_CUDA; }
+  }
+  return PS_OK;
+}
+
+int push_checked(ps_service* s, int job, int block, int worker, const void* ptr, Block** out) {
+  const int bi = find_block(s, job, block);
+  if (bi < 0 || !ptr) return PS_ERR_BAD_ARG;
+  Block& b = s->blocks[bi];
+  const Job& j = s->jobs[b.job];
+  if (worker < 0 || worker >= j.d.num_workers) return PS_ERR_BAD_ARG;
+  if (reinterpret_cast<uintptr_t>(ptr) & (j.grad_esize() - 1)) return PS_ERR_ALIGN;
+  if (b.pushed[worker]) return PS_ERR_DUPLICATE;
+  *out = &b;
+  return PS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes_per_ctx) {
+  if (!out || num_contexts < 1 || num_contexts > 1024 || device < PS_DEVICE_NONE) return PS_ERR_BAD_ARG;
+  *out = nullptr;
+  ps_service* s = new (std::nothrow) ps_service();
+  if (!s) return PS_ERR_NOMEM;
+  s->device = device;
+  s->ctxs.resize(num_contexts);
+  for (auto& c : s->ctxs) c.arena.reset(arena_bytes_per_ctx);
+  if (device >= 0) {
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->num_sms, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess)
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&s->occ_ctas, ps_aggregate_ldg_kernel, kThreads, 0);
+    for (int c = 0; e == cudaSuccess && c < num_contexts; ++c) {
+      void* base = nullptr;
+      e = cudaMalloc(&base, s->ctxs[c].arena.capacity() ? s->ctxs[c].arena.capacity() : Arena::kAlign);
+      s->ctxs[c].base = static_cast<char*>(base);
+    }
+    if (e != cudaSuccess) {
+      const bool oom = (e == cudaErrorMemoryAllocation);
+      for (auto& c : s->ctxs) if (c.base) cudaFree(c.base);
+      cudaGetLastError();
+      delete s;
+      return oom ? PS_ERR_NOMEM : PS_ERR_CUDA;
+    }
+  }
+  *out = s;
+  return PS_OK;
+}
+
+int ps_destroy(ps_service* s) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  if (has_device(s)) {
+    cudaSetDevice(s->device);
+    cudaDeviceSynchronize();
+    for (auto& b : s->blocks) {
+      if (b.mig_event) cudaEventDestroy(b.mig_event);
+      if (b.staging) cudaFree(b.staging);
+    }
+    for (auto& sl : s->slots) {
+      if (sl.host) cudaFreeHost(sl.host);
+      if (sl.dev) cudaFree(sl.dev);
+      if (sl.partials) cudaFree(sl.partials);
+      if (sl.done) cudaEventDestroy(sl.done);
+    }
+    for (auto& c : s->ctxs) if (c.base) cudaFree(c.base);
+    if (s->jobs_dev) cudaFree(s->jobs_dev);
+    if (s->stats_dev) cudaFree(s->stats_dev);
+  }
+  s->magic = 0;
+  delete s;
+  return PS_OK;
+}
+
+int ps_register_job(ps_service* s, const ps_job_desc* d, int* job_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (!d || !job_out) return PS_ERR_BAD_ARG;
+  if (d->opt != PS_SGD && d->opt != PS_ADAM) return PS_ERR_BAD_ARG;
+  if (d->grad_dtype != PS_F32 && d->grad_dtype != PS_BF16) return PS_ERR_BAD_ARG;
+  if (d->num_workers < 1 || d->num_workers > PS_MAX_WORKERS) return PS_ERR_BAD_ARG;
+  const int id = (int)s->jobs.size();
+  if (has_device(s)) {
+    PS_CUDA(s, cudaSetDevice(s->device));
+    int rc = grow_dev(s, &s->jobs_dev, &s->jobs_dev_cap, (size_t)id + 1, false);
+    if (rc) return rc;
+    PsJobDev jd;
+    std::memset(&jd, 0, sizeof jd);
+    jd.opt = d->opt; jd.grad_dtype = d->grad_dtype; jd.W = d->num_workers;
+    jd.lr = d->lr; jd.mom = d->momentum; jd.wd = d->weight_decay;
+    jd.b1 = d->beta1; jd.b2 = d->beta2;
+    jd.omb1 = 1.0f - d->beta1;
+    jd.omb2 = 1.0f - d->beta2;
+    jd.eps = d->eps; jd.gs = d->grad_scale;
+    PS_CUDA(s, cudaMemcpy(s->jobs_dev + id, &jd, sizeof jd, cudaMemcpyHostToDevice));
+  }
+  Job j;
+  j.d = *d;
+  s->jobs.push_back(j);
+  *job_out = id;
+  return PS_OK;
+}
+
+int ps_register_block(ps_service* s, int job, int block, size_t nelem, int ctx, const float* init) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (job < 0 || job >= (int)s->jobs.size() || block < 0 || block >= (1 << 26)) return PS_ERR_BAD_ARG;
+  if (nelem == 0 || nelem > ((size_t)1 << 40) || ctx < 0 || ctx >= (int)s->ctxs.size()) return PS_ERR_BAD_ARG;
+  Job& j = s->jobs[job];
+  if (block < (int)j.block_of_id.size() && j.block_of_id[block] >= 0) return PS_ERR_DUPLICATE;
+  Block b;
+  b.job = job; b.id = block; b.nelem = nelem; b.ctx = ctx;
+  b.sec = Arena::round_up(nelem * sizeof(float));
+  b.bytes = b.sec * (1 + j.nstate());
+  b.pushed.assign(j.d.num_workers, nullptr);
+  b.stat_idx = (unsigned int)s->blocks.size();
+  if (has_device(s)) PS_CUDA(s, cudaSetDevice(s->device));
+  int rc = arena_alloc(s, ctx, b.bytes, &b.off);
+  if (rc) return rc;
+  if (has_device(s)) {
+    rc = grow_dev(s, &s->stats_dev, &s->stats_dev_cap, s->blocks.size() + 1, true);
+    cudaError_t e = cudaSuccess;
+    if (!rc) {
+      char* base = s->ctxs[ctx].base + b.off;
+      e = cudaMemset(base, 0, b.bytes);
+      if (e == cudaSuccess && init) e = cudaMemcpy(base, init, nelem * sizeof(float), cudaMemcpyDefault);
+      if (e != cudaSuccess) { s->cuda_err = cudaGetErrorString(e); rc = PS_ERR_CUDA; }
+    }
+    if (rc) { s->ctxs[ctx].arena.release(b.off, b.bytes); return rc; }
+  }
+  if (block >= (int)j.block_of_id.size()) j.block_of_id.resize(block + 1, -1);
+  j.block_of_id[block] = (int)s->blocks.size();
+  s->blocks.push_back(std::move(b));
+  return PS_OK;
+}
+
+int ps_push(ps_service* s, int job, int block, int worker, const void* ptr) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  Block* b = nullptr;
+  int rc = push_checked(s, job, block, worker, ptr, &b);
+  if (rc) return rc;
+  b->pushed[worker] = ptr;
+  b->npushed++;
+  return PS_OK;
+}
+
+int ps_push_batch(ps_service* s, int n, const int* jobs, const int* blocks, const int* workers,
+                  const void* const* ptrs) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (n < 0 || (n > 0 && (!jobs || !blocks || !workers || !ptrs))) return PS_ERR_BAD_ARG;
+  int rc = PS_OK, done = 0;
+  for (; done < n; ++done) {
+    Block* b = nullptr;
+    rc = push_checked(s, jobs[done], blocks[done], workers[done], ptrs[done], &b);
+    if (rc) break;
+    b->pushed[workers[done]] = ptrs[done];
+    b->npushed++;
+  }
+  if (rc) {   // roll back: all-or-nothing
+    for (int i = 0; i < done; ++i) {
+      Block& b = s->blocks[find_block(s, jobs[i], blocks[i])];
+      b.pushed[workers[i]] = nullptr;
+      b.npushed--;
+    }
+  }
+  return rc;
+}
+
+int ps_push_host(ps_service* s, int job, int block, int worker, const void* host_ptr, void* stream) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  Block* b = nullptr;
+  int rc = push_checked(s, job, block, worker, host_ptr, &b);
+  if (rc) return rc;
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  PS_CUDA(s, cudaSetDevice(s->device));
+  const Job& j = s->jobs[b->job];
+  if (!b->staging) {
+    b->staging_row = Arena::round_up(b->nelem * j.grad_esize());
+    cudaError_t e = cudaMalloc(&b->staging, b->staging_row * j.d.num_workers);
+    if (e != cudaSuccess) {
+      b->staging = nullptr;
+      cudaGetLastError();
+      if (e == cudaErrorMemoryAllocation) return PS_ERR_NOMEM;
+      s->cuda_err = cudaGetErrorString(e);
+      return PS_ERR_CUDA;
+    }
+  }
+  char* dst = static_cast<char*>(b->staging) + (size_t)worker * b->staging_row;
+  PS_CUDA(s, cudaMemcpyAsync(dst, host_ptr, b->nelem * j.grad_esize(), cudaMemcpyHostToDevice,
+                             static_cast<cudaStream_t>(stream)));
+  b->pushed[worker] = dst;
+  b->npushed++;
+  return PS_OK;
+}
+
+int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  std::vector<int> idx;
+  int rc = validate_ready(s, ready, n_ready, &idx);
+  if (rc) return rc;
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  if (idx.empty()) return PS_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  PS_CUDA(s, cudaSetDevice(s->device));
+  Plan plan;
+  rc = build_plan(s, idx, &plan);
+  if (rc) return rc;
+  Slot* sl = nullptr;
+  rc = acquire_slot(s, plan.bytes.size(), plan.total_chunks, &sl);
+  if (rc) return rc;
+  for (int bi : idx) {
+    rc = order_after_block(s, s->blocks[bi], stream);
+    if (rc) return rc;
+  }
+  std::memcpy(sl->host, plan.bytes.data(), plan.bytes.size());
+  PS_CUDA(s, cudaMemcpyAsync(sl->dev, sl->host, plan.bytes.size(), cudaMemcpyHostToDevice, stream));
+  const int grid = (int)std::min<unsigned long long>(plan.total_chunks, (unsigned long long)grid_cap(s));
+  ps_aggregate_ldg_kernel<<<grid, kThreads, 0, stream>>>(sl->dev, s->jobs_dev, s->stats_dev, sl->partials);
+  PS_CUDA(s, cudaGetLastError());
+  PS_CUDA(s, cudaEventRecord(sl->done, stream));
+  sl->inflight = true;
+  const int slot_index = (int)(sl - s->slots);
+  s->next_slot = (s->next_slot + 1) % kSlots;
+  s->launches++;
+  s->last_grid = grid;
+  s->last_block = kThreads;
+  s->last_kernel = "ldg";
+  for (int bi : idx) {
+    Block& b = s->blocks[bi];
+    b.step++;
+    std::fill(b.pushed.begin(), b.pushed.end(), nullptr);
+    b.npushed = 0;
+    b.last_slot = slot_index;
+    b.last_slot_gen = sl->gen;
+  }
+  return PS_OK;
+}
+
+int ps_plan(ps_service* s, const ps_task* ready, int n_ready, ps_chunk_info* out, size_t cap, size_t* n_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  std::vector<int> idx;
+  int rc = validate_ready(s, ready, n_ready, &idx);
+  if (rc) return rc;
+  Plan plan;
+  if (!idx.empty()) {
+    rc = build_plan(s, idx, &plan);
+    if (rc) return rc;
+  }
+  if (n_out) *n_out = plan.total_chunks;
+  if (!out || idx.empty()) return PS_OK;
+  const unsigned char* base = plan.bytes.data();
+  const PsTableHdr* h = reinterpret_cast<const PsTableHdr*>(base);
+  const PsTaskDev* tasks = reinterpret_cast<const PsTaskDev*>(base + h->tasks_off);
+  size_t k = 0;
+  for (unsigned int t = 0; t < h->n_tasks && k < cap; ++t) {
+    const Block& b = s->blocks[plan.order[t]];
+    for (unsigned int c = 0; c < tasks[t].nchunks && k < cap; ++c, ++k) {
+      ps_chunk_info& ci = out[k];
+      ci.job = b.job;
+      ci.block = b.id;
+      ci.elem_begin = (unsigned long long)c * h->chunk_elems;
+      ci.elem_count = std::min<unsigned long long>(h->chunk_elems, tasks[t].nelem - ci.elem_begin);
+      ci.num_workers = s->jobs[b.job].d.num_workers;
+      ci.vector_path = (int)tasks[t].vec_ok;
+    }
+  }
+  return PS_OK;
+}
+
+int ps_pull(ps_service* s, int job, int block, const float** out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  const int bi = find_block(s, job, block);
+  if (bi < 0 || !out) return PS_ERR_BAD_ARG;
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  *out = blk_p(s, s->blocks[bi]);
+  return PS_OK;
+}
+
+int ps_pull_host(ps_service* s, int job, int block, float* dst, void* stream_) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  const int bi = find_block(s, job, block);
+  if (bi < 0 || !dst) return PS_ERR_BAD_ARG;
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  PS_CUDA(s, cudaSetDevice(s->device));
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  Block& b = s->blocks[bi];
+  int rc = order_after_block(s, b, stream);
+  if (rc) return rc;
+  PS_CUDA(s, cudaMemcpyAsync(dst, blk_p(s, b), b.nelem * sizeof(float), cudaMemcpyDeviceToHost, stream));
+  return PS_OK;
+}
+
+int ps_migrate_block(ps_service* s, int job, int block, int dst_ctx, void* stream_) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  const int bi = find_block(s, job, block);
+  if (bi < 0 || dst_ctx < 0 || dst_ctx >= (int)s->ctxs.size()) return PS_ERR_BAD_ARG;
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  Block& b = s->blocks[bi];
+  if (b.ctx == dst_ctx) return PS_OK;
+  PS_CUDA(s, cudaSetDevice(s->device));
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (b.mig_pending) {   // a second move before the first copy landed: let it land
+    PS_CUDA(s, cudaEventSynchronize(b.mig_event));
+    b.mig_pending = false;
+    int rc0 = reap_frees(s, false);
+    if (rc0) return rc0;
+  }
+  size_t noff = 0;
+  int rc = arena_alloc(s, dst_ctx, b.bytes, &noff);
+  if (rc) return rc;
+  if (!b.mig_event) {
+    cudaError_t e = cudaEventCreateWithFlags(&b.mig_event, cudaEventDisableTiming);
+    if (e != cudaSuccess) {
+      s->ctxs[dst_ctx].arena.release(noff, b.bytes);
+      s->cuda_err = cudaGetErrorString(e);
+      return PS_ERR_CUDA;
+    }
+  }
+  rc = order_after_block(s, b, stream);
+  cudaError_t e = cudaSuccess;
+  if (!rc) {
+    // parameters, optimizer state (one contiguous range); the step counter is host state
+    e = cudaMemcpyAsync(s->ctxs[dst_ctx].base + noff, s->ctxs[b.ctx].base + b.off, b.bytes,
+                        cudaMemcpyDeviceToDevice, stream);
+    if (e == cudaSuccess) e = cudaEventRecord(b.mig_event, stream);
+    if (e != cudaSuccess) { s->cuda_err = cudaGetErrorString(e); rc = PS_ERR_CUDA; }
+  }
+  if (rc) { s->ctxs[dst_ctx].arena.release(noff, b.bytes); return rc; }
+  s->pending_free.push_back(PendingFree{b.ctx, b.off, b.bytes, b.mig_event, bi});
+  b.ctx = dst_ctx;
+  b.off = noff;
+  b.mig_pending = true;
+  return PS_OK;
+}
+
+int ps_block_stats(ps_service* s, int job, int block, double* sq_out, unsigned long long* step_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  const int bi = find_block(s, job, block);
+  if (bi < 0) return PS_ERR_BAD_ARG;
+  Block& b = s->blocks[bi];
+  if (step_out) *step_out = b.step;
+  if (!sq_out) return PS_OK;
+  *sq_out = 0.0;
+  if (!has_device(s) || b.last_slot < 0) return PS_OK;
+  PS_CUDA(s, cudaSetDevice(s->device));
+  Slot& sl = s->slots[b.last_slot];
+  if (sl.inflight && sl.gen == b.last_slot_gen) PS_CUDA(s, cudaEventSynchronize(sl.done));
+  PsStat st;
+  PS_CUDA(s, cudaMemcpy(&st, s->stats_dev + b.stat_idx, sizeof st, cudaMemcpyDeviceToHost));
+  *sq_out = st.sqnorm;
+  return PS_OK;
+}
+
+int ps_block_state(ps_service* s, int job, int block, const float** s0, const float** s1, int* ctx_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  const int bi = find_block(s, job, block);
+  if (bi < 0) return PS_ERR_BAD_ARG;
+  Block& b = s->blocks[bi];
+  if (ctx_out) *ctx_out = b.ctx;
+  if (s0) *s0 = has_device(s) ? blk_s0(s, b) : nullptr;
+  if (s1) *s1 = has_device(s) ? blk_s1(s, b) : nullptr;
+  return PS_OK;
+}
+
+int ps_set_option(ps_service* s, int option, long long value) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  switch (option) {
+    case PS_OPT_CHUNK_ELEMS:
+      if (value < 0 || value > (long long)kMaxChunk || (value % 1024) != 0) return PS_ERR_BAD_ARG;
+      s->opt_chunk = value;
+      return PS_OK;
+    case PS_OPT_CTAS_PER_SM:
+      if (value < 0 || value > 32) return PS_ERR_BAD_ARG;
+      s->opt_ctas = value;
+      return PS_OK;
+    case PS_OPT_SORT_TASKS:
+      s->opt_sort = value ? 1 : 0;
+      return PS_OK;
+    case PS_OPT_KERNEL:
+      if (value < 0 || value > 1) return PS_ERR_BAD_ARG;
+      s->opt_kernel = value;
+      return PS_OK;
+    default:
+      return PS_ERR_BAD_ARG;
+  }
+}
+
+int ps_get_option(ps_service* s, int option, long long* out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (!out) return PS_ERR_BAD_ARG;
+  switch (option) {
+    case PS_OPT_CHUNK_ELEMS: *out = s->opt_chunk; return PS_OK;
+    case PS_OPT_CTAS_PER_SM: *out = s->opt_ctas; return PS_OK;
+    case PS_OPT_SORT_TASKS: *out = s->opt_sort; return PS_OK;
+    case PS_OPT_KERNEL: *out = s->opt_kernel; return PS_OK;
+    default: return PS_ERR_BAD_ARG;
+  }
+}
+
+int ps_arena_info(ps_service* s, int ctx, size_t* used_out, size_t* largest_free_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (ctx < 0 || ctx >= (int)s->ctxs.size()) return PS_ERR_BAD_ARG;
+  if (has_device(s)) {
+    int rc = reap_frees(s, false);
+    if (rc) return rc;
+  }
+  if (used_out) *used_out = s->ctxs[ctx].arena.used();
+  if (largest_free_out) *largest_free_out = s->ctxs[ctx].arena.largest_free();
+  return PS_OK;
+}
+
+int ps_launch_info(ps_service* s, unsigned long long* launches, int* grid, int* block, const char** name) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (launches) *launches = s->launches;
+  if (grid) *grid = s->last_grid;
+  if (block) *block = s->last_block;
+  if (name) *name = s->last_kernel;
+  return PS_OK;
+}
+
+const char* ps_strerror(int status) {
+  switch (status) {
+    case PS_OK: return "ok";
+    case PS_ERR_BAD_HANDLE: return "bad service handle";
+    case PS_ERR_BAD_ARG: return "bad argument";
+    case PS_ERR_DUPLICATE: return "duplicate block, push or task";
+    case PS_ERR_NOT_READY: return "a listed task has fewer than W pushes";
+    case PS_ERR_ALIGN: return "gradient pointer not aligned to its element size";
+    case PS_ERR_NOMEM: return "out of arena, device or host memory";
+    case PS_ERR_CUDA: return "CUDA runtime error";
+    case PS_ERR_NO_DEVICE: return "service has no device (planning only)";
+    default: return "unknown status";
+  }
+}
+
+const char* ps_last_cuda_error(ps_service* s) { return alive(s) ? s->cuda_err.c_str() : ""; }
+
+const char* ps_version(void) { return "ps_b200 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,127 @@
+"""Shared test plumbing: drives the CUDA service and the CPU oracle with the
+same seeded inputs and compares them element by element."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import aggregator as A
+from paper_2204_03211_b200 import binding as B
+from workload import configs, generate
+
+TOL = 1e-6      # max |delta| <= TOL * (1 + |ref|) for fp32 state (spec tolerance; bit-equality expected)
+
+
+def to_np(t: torch.Tensor) -> np.ndarray:
+    t = t.detach().cpu().contiguous()
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).numpy().view(np.uint16)
+    return t.numpy()
+
+
+def oracle_hp(job: configs.JobSpec) -> A.HParams:
+    return A.HParams(**job.hparams())
+
+
+def assert_close(got: np.ndarray, ref: np.ndarray, what: str, tol: float = TOL):
+    assert got.shape == ref.shape, what
+    err = np.abs(got.astype(np.float64) - ref.astype(np.float64))
+    bound = tol * (1.0 + np.abs(ref.astype(np.float64)))
+    bad = err > bound
+    assert not bad.any(), "%s: %d/%d elements off, max err %.3e at %d" % (
+        what, int(bad.sum()), bad.size, float(err.max()), int(err.argmax()))
+
+
+class Pair:
+    """One CUDA service and one oracle fed the same registrations and pushes."""
+
+    def __init__(self, cfg: configs.Config, device: int = 0, arena_bytes: int | None = None, nthreads: int = 0):
+        self.cfg = cfg
+        self.dev = torch.device("cuda", device)
+        need = sum(3 * (4 * b.nelem + 256) for j in cfg.jobs for b in j.blocks) + (1 << 20)
+        self.svc = B.Service(device, cfg.num_contexts, arena_bytes or need)
+        self.ora = A.OracleAggregator(cfg.num_contexts, nthreads)
+        self.keep = []          # gradient tensors of the iteration in flight
+        for j, job in enumerate(cfg.jobs):
+            jid = self.svc.register_job(**job.hparams())
+            assert jid == self.ora.register_job(oracle_hp(job)) == j
+            p0 = generate.init_params(cfg, j)
+            for b in job.blocks:
+                init = p0[b.job_offset:b.job_offset + b.nelem].contiguous()
+                ctx = configs.initial_context(cfg, j, b.block)
+                self.svc.register_block(j, b.block, b.nelem, ctx, init)
+                self.ora.register_block(j, b.block, b.nelem, ctx, init.numpy())
+
+    def close(self):
+        self.svc.close()
+
+    def push_iteration(self, it: int, jobs=None):
+        """Generates iteration `it`'s gradients on the CPU and pushes every
+        block of the given jobs to both sides."""
+        self.keep = []
+        for j, job in enumerate(self.cfg.jobs):
+            if jobs is not None and j not in jobs:
+                continue
+            slab = generate.grad_slab(self.cfg, j, it)
+            dslab = slab.to(self.dev)
+            self.keep.append((slab, dslab))
+            host = to_np(slab)
+            esz = dslab.element_size()
+            for b in job.blocks:
+                for w in range(job.num_workers):
+                    self.svc.push(j, b.block, w, dslab.data_ptr() + (w * job.num_params + b.job_offset) * esz)
+                    self.ora.push(j, b.block, w, host[w, b.job_offset:b.job_offset + b.nelem])
+
+    def aggregate(self, ready, stream=None):
+        self.svc.aggregate(ready, stream)
+        self.ora.aggregate(list(ready))
+
+    def migrate(self, job, block, dst, stream=None):
+        self.svc.migrate_block(job, block, dst, stream)
+        self.ora.migrate_block(job, block, dst)
+
+    def gpu_block(self, j: int, b: int):
+        n = self.cfg.jobs[j].blocks[b].nelem
+        s0, s1, ctx = self.svc.block_state(j, b)
+        torch.cuda.synchronize(self.dev)
+        p = self.svc.view(self.svc.pull(j, b), n).cpu().numpy()
+        a = self.svc.view(s0, n).cpu().numpy()
+        v = self.svc.view(s1, n).cpu().numpy() if s1 else None
+        return p, a, v, ctx
+
+    def compare(self, sq_rtol: float = 1e-5, exact: bool = True):
+        worst = 0.0
+        for j, job in enumerate(self.cfg.jobs):
+            for b in job.blocks:
+                p, a, v, ctx = self.gpu_block(j, b.block)
+                rp = self.ora.pull(j, b.block)
+                ra, rv = self.ora.state(j, b.block)
+                tag = "%s job %d block %d" % (self.cfg.name, j, b.block)
+                assert_close(p, rp, tag + " params")
+                assert_close(a, ra, tag + " state0")
+                if rv is not None:
+                    assert_close(v, rv, tag + " state1")
+                if exact:
+                    assert np.array_equal(p, rp) and np.array_equal(a, ra), tag + " not bit-identical"
+                    if rv is not None:
+                        assert np.array_equal(v, rv), tag + " state1 not bit-identical"
+                assert ctx == self.ora.blocks[(j, b.block)].ctx, tag + " context"
+                sq, step = self.svc.block_stats(j, b.block)
+                rsq, rstep = self.ora.block_stats(j, b.block)
+                assert step == rstep, tag + " step"
+                assert abs(sq - rsq) <= sq_rtol * abs(rsq) + 1e-300, tag + " sqnorm %r vs %r" % (sq, rsq)
+                worst = max(worst, float(np.max(np.abs(p.astype(np.float64) - rp))))
+        return worst
+
+
+def tiny_config(sizes, W, opt=configs.SGD, grad_dtype=configs.F32, seed=123, **kw) -> configs.Config:
+    """One job whose blocks have the given element counts."""
+    from workload import shapes
+    tensors = [shapes.Tensor("t%d" % i, (n,), i) for i, n in enumerate(sizes)]
+    blocks = shapes.cut_blocks(tensors, keep_whole=lambda t: True)
+    base = dict(lr=0.1, momentum=0.9, weight_decay=1e-4, grad_std=1e-2)
+    if opt == configs.ADAM:
+        base = dict(lr=1e-3, momentum=0.0, weight_decay=1e-2, grad_std=1e-2)
+    base.update(kw)
+    job = configs.JobSpec("tiny", "tiny", tensors, blocks, W, opt=opt, grad_dtype=grad_dtype, **base)
+    return configs.Config("tiny", seed, 3, [job])

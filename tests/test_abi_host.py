@@ -1,0 +1,200 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every symbol the
+public header declares, and its host logic (registry, push bookkeeping, task
+packing, arena) behaves.  No kernel is launched: the services here are
+planning-only (PS_DEVICE_NONE) and every compute entry point must refuse."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2204_03211_b200 import binding as B, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "ps_b200.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ps_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(B.LIB_PATH)
+    names = _declared()
+    assert {"ps_create", "ps_register_job", "ps_register_block", "ps_push", "ps_aggregate", "ps_pull",
+            "ps_migrate_block"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(B._SIGNATURES), "binding and header disagree"
+
+
+def test_struct_layouts_match_the_header():
+    assert ctypes.sizeof(B.ps_job_desc) == 40 and ctypes.sizeof(B.ps_task) == 8
+    assert ctypes.sizeof(B.ps_chunk_info) == 32
+
+
+def test_strerror_and_version():
+    assert B.ps_strerror(0) == "ok" and "W" in B.ps_strerror(B.PS_ERR_NOT_READY)
+    assert "sm_100a" in B.ps_version()
+
+
+def test_no_device_means_loud_failure_not_fallback():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device exists here")
+    with pytest.raises(B.PsError) as e:
+        B.ps_create(0, 1, 1 << 20)
+    assert e.value.status in (B.PS_ERR_CUDA, B.PS_ERR_NOMEM)
+
+
+def _svc(**kw):
+    return B.Service(device=B.PS_DEVICE_NONE, num_contexts=kw.get("ctxs", 2), arena_bytes_per_ctx=kw.get("arena", 1 << 30))
+
+
+def _status(fn, *a):
+    try:
+        fn(*a)
+    except B.PsError as e:
+        return e.status
+    return 0
+
+
+def test_registration_errors():
+    s = _svc()
+    assert _status(s.register_job, B.PS_SGD, B.PS_F32, 0) == B.PS_ERR_BAD_ARG
+    assert _status(s.register_job, 7) == B.PS_ERR_BAD_ARG
+    assert _status(s.register_job, B.PS_SGD, 3, 2) == B.PS_ERR_BAD_ARG
+    assert _status(s.register_job, B.PS_SGD, B.PS_F32, B.PS_MAX_WORKERS + 1) == B.PS_ERR_BAD_ARG
+    j = s.register_job(num_workers=2)
+    assert j == 0 and s.register_job(num_workers=3) == 1
+    s.register_block(j, 4, 100, 1)
+    assert _status(s.register_block, j, 4, 100, 0) == B.PS_ERR_DUPLICATE
+    assert _status(s.register_block, j, 5, 0, 0) == B.PS_ERR_BAD_ARG
+    assert _status(s.register_block, j, 5, 10, 2) == B.PS_ERR_BAD_ARG
+    assert _status(s.register_block, 9, 0, 10, 0) == B.PS_ERR_BAD_ARG
+    assert _status(s.register_block, j, -1, 10, 0) == B.PS_ERR_BAD_ARG
+    assert s.block_state(j, 4)[2] == 1
+    assert _status(B.ps_destroy, None) == B.PS_ERR_BAD_HANDLE
+
+
+def test_push_bookkeeping_and_ready_list_validation():
+    s = _svc()
+    j = s.register_job(num_workers=2)
+    k = s.register_job(num_workers=1, grad_dtype=B.PS_BF16)
+    s.register_block(j, 0, 5000)
+    s.register_block(k, 0, 300)
+    assert _status(s.push, j, 0, 2, 4096) == B.PS_ERR_BAD_ARG
+    assert _status(s.push, j, 1, 0, 4096) == B.PS_ERR_BAD_ARG
+    assert _status(s.push, j, 0, 0, 0) == B.PS_ERR_BAD_ARG
+    assert _status(s.push, j, 0, 0, 4098) == B.PS_ERR_ALIGN        # fp32 needs 4-byte alignment
+    assert _status(s.push, k, 0, 0, 4097) == B.PS_ERR_ALIGN        # bf16 needs 2-byte alignment
+    s.push(k, 0, 0, 4098)
+    s.push(j, 0, 0, 4096)
+    assert _status(s.push, j, 0, 0, 4096) == B.PS_ERR_DUPLICATE
+    assert _status(s.plan, [(j, 0)]) == B.PS_ERR_NOT_READY
+    assert _status(s.plan, [(k, 0), (j, 0)]) == B.PS_ERR_NOT_READY
+    s.push(j, 0, 1, 8192)
+    assert _status(s.plan, [(j, 0), (j, 0)]) == B.PS_ERR_DUPLICATE
+    assert _status(s.plan, [(j, 3)]) == B.PS_ERR_BAD_ARG
+    assert len(s.plan([(j, 0), (k, 0)])) >= 2
+    # compute entry points refuse on a planning-only service
+    assert _status(s.aggregate, [(j, 0)]) == B.PS_ERR_NO_DEVICE
+    assert _status(s.pull, j, 0) == B.PS_ERR_NO_DEVICE
+    assert _status(s.migrate_block, j, 0, 1) == B.PS_ERR_NO_DEVICE
+    assert _status(s.push_host, k, 0, 0, 4096) == B.PS_ERR_DUPLICATE   # validation comes first
+    assert s.block_stats(j, 0) == (0.0, 0)
+    assert s.plan([]) == []
+
+
+def test_push_batch_is_all_or_nothing():
+    s = _svc()
+    j = s.register_job(num_workers=2)
+    s.register_block(j, 0, 64)
+    s.register_block(j, 1, 64)
+    jobs = np.array([j, j, j, j], np.int32)
+    blocks = np.array([0, 0, 1, 1], np.int32)
+    workers = np.array([0, 1, 0, 0], np.int32)           # last one is a duplicate
+    ptrs = np.array([4096, 8192, 12288, 16384], np.uint64)
+    assert _status(s.push_batch, jobs, blocks, workers, ptrs) == B.PS_ERR_DUPLICATE
+    assert _status(s.plan, [(j, 0)]) == B.PS_ERR_NOT_READY    # rolled back
+    workers[3] = 1
+    s.push_batch(jobs, blocks, workers, ptrs)
+    assert len(s.plan([(j, 0), (j, 1)])) == 2
+
+
+@pytest.mark.parametrize("chunk", [0, 1024, 4096, 1 << 20])
+def test_plan_covers_every_element_exactly_once(chunk):
+    s = _svc()
+    s.set_option(B.PS_OPT_CHUNK_ELEMS, chunk)
+    rng = np.random.default_rng(chunk)
+    sizes = {}
+    ready = []
+    for W in (1, 2, 16):
+        j = s.register_job(num_workers=W, opt=B.PS_ADAM if W == 16 else B.PS_SGD)
+        for b in range(6):
+            n = int(rng.choice([1, 3, 1023, 1024, 1025, 5000, 1 << 20, (1 << 20) + 1, 2_359_296]))
+            s.register_block(j, b, n)
+            sizes[(j, b)] = (n, W)
+            for w in range(W):
+                s.push(j, b, w, 4096 * (1 + w) + (4 if (b == 5 and w == 0) else 0))
+            ready.append((j, b))
+    plan = s.plan(ready)
+    seen = {k: [] for k in sizes}
+    for c in plan:
+        n, W = sizes[(c.job, c.block)]
+        assert c.num_workers == W and c.elem_count > 0
+        assert c.vector_path == (0 if c.block == 5 else 1)
+        seen[(c.job, c.block)].append((c.elem_begin, c.elem_count))
+    for k, (n, W) in sizes.items():
+        spans = sorted(seen[k])
+        pos = 0
+        for b, cnt in spans:
+            assert b == pos and b % 1024 == 0        # chunk starts keep 128-bit alignment
+            pos += cnt
+        assert pos == n
+    # chunks of one task are contiguous in claim order
+    keys = [(c.job, c.block) for c in plan]
+    assert len([1 for a, b in zip(keys, keys[1:]) if a != b]) == len(sizes) - 1
+
+
+def test_heaviest_chunks_are_claimed_first_unless_sorting_is_off():
+    s = _svc()
+    light = s.register_job(num_workers=1)
+    heavy = s.register_job(num_workers=16)
+    for j, W in ((light, 1), (heavy, 16)):
+        s.register_block(j, 0, 1 << 16)
+        for w in range(W):
+            s.push(j, 0, w, 4096)
+    s.set_option(B.PS_OPT_CHUNK_ELEMS, 4096)
+    assert s.plan([(light, 0), (heavy, 0)])[0].job == heavy
+    s.set_option(B.PS_OPT_SORT_TASKS, 0)
+    assert s.plan([(light, 0), (heavy, 0)])[0].job == light
+
+
+def test_options_validate():
+    s = _svc()
+    assert _status(s.set_option, B.PS_OPT_CHUNK_ELEMS, 1000) == B.PS_ERR_BAD_ARG
+    assert _status(s.set_option, B.PS_OPT_CHUNK_ELEMS, (1 << 20) + 1024) == B.PS_ERR_BAD_ARG
+    assert _status(s.set_option, 99, 1) == B.PS_ERR_BAD_ARG
+    s.set_option(B.PS_OPT_CTAS_PER_SM, 2)
+    assert s.get_option(B.PS_OPT_CTAS_PER_SM) == 2 and s.get_option(B.PS_OPT_SORT_TASKS) == 1
+
+
+def test_arena_accounting_and_exhaustion():
+    s = _svc(ctxs=1, arena=1 << 20)
+    j = s.register_job(num_workers=1, opt=B.PS_ADAM)
+    used0, free0 = s.arena_info(0)
+    assert used0 == 0 and free0 == 1 << 20
+    s.register_block(j, 0, 1000)                     # 3 ranges of 4000 B -> 3 * 4096
+    assert s.arena_info(0)[0] == 3 * 4096
+    assert _status(s.register_block, j, 1, 100_000, 0) == B.PS_ERR_NOMEM
+    assert s.arena_info(0)[0] == 3 * 4096            # failed registration left nothing behind
+    s.register_block(j, 1, 80_000)
+    assert s.arena_info(0)[0] == 3 * 4096 + 3 * 320_000

@@ -1,0 +1,158 @@
+"""CUDA path vs CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import Pair, tiny_config, to_np, assert_close
+from paper_2204_03211_b200 import binding as B
+from workload import configs, generate
+
+pytestmark = pytest.mark.gpu
+
+ODD_SIZES = [1, 3, 4, 5, 127, 1024, 4097, 12289, 70001]
+
+
+@pytest.mark.parametrize("opt,dt", [(configs.SGD, configs.F32), (configs.ADAM, configs.F32),
+                                    (configs.SGD, configs.BF16), (configs.ADAM, configs.BF16)])
+@pytest.mark.parametrize("W", [1, 2, 5, 8, 33])
+def test_odd_sizes_bit_exact(opt, dt, W):
+    cfg = tiny_config(ODD_SIZES, W, opt=opt, grad_dtype=dt)
+    pair = Pair(cfg)
+    try:
+        every = configs.rounds_all(cfg)[0]
+        for it in range(3):
+            pair.push_iteration(it)
+            pair.aggregate(every)
+            pair.compare()
+    finally:
+        pair.close()
+
+
+@pytest.mark.parametrize("chunk", [1024, 2048, 8192, 65536])
+def test_chunk_size_and_order_invariance(chunk):
+    cfg = tiny_config([5, 40000, 1024, 300001, 77], 4)
+    pair = Pair(cfg)
+    try:
+        pair.svc.set_option(B.PS_OPT_CHUNK_ELEMS, chunk)
+        pair.svc.set_option(B.PS_OPT_SORT_TASKS, chunk % 2048 == 0)
+        order = [(0, 3), (0, 0), (0, 4), (0, 1), (0, 2)]
+        for it in range(2):
+            pair.push_iteration(it)
+            pair.aggregate(order)
+        pair.compare()
+    finally:
+        pair.close()
+
+
+def test_unaligned_shards_take_scalar_path_same_bits():
+    cfg = tiny_config([4099, 600], 3)
+    pair = Pair(cfg)
+    try:
+        job = cfg.jobs[0]
+        slab = generate.grad_slab(cfg, 0, 0)
+        host = to_np(slab)
+        # device copy shifted by one float: every shard pointer is only 4-byte aligned
+        dbuf = torch.empty(slab.numel() + 1, dtype=torch.float32, device="cuda")
+        dbuf[1:].copy_(slab.reshape(-1))
+        base = dbuf.data_ptr() + 4
+        for b in job.blocks:
+            for w in range(3):
+                off = w * job.num_params + b.job_offset
+                pair.svc.push(0, b.block, w, base + 4 * off)
+                pair.ora.push(0, b.block, w, host[w, b.job_offset:b.job_offset + b.nelem])
+        plan = pair.svc.plan([(0, 0), (0, 1)])
+        assert any(c.vector_path == 0 for c in plan)
+        pair.aggregate([(0, 0), (0, 1)])
+        pair.compare()
+        with pytest.raises(B.PsError) as e:
+            pair.svc.push(0, 0, 0, base + 2)
+        assert e.value.status == B.PS_ERR_ALIGN
+    finally:
+        pair.close()
+
+
+def test_c1_ten_iterations():
+    cfg = configs.c1()
+    pair = Pair(cfg)
+    try:
+        every = configs.rounds_all(cfg)[0]
+        for it in range(cfg.iterations):
+            pair.push_iteration(it)
+            pair.aggregate(every)
+            if it in (0, cfg.iterations - 1):
+                pair.compare()
+    finally:
+        pair.close()
+
+
+def test_results_repeat_bit_for_bit_across_runs():
+    outs = []
+    for _ in range(2):
+        cfg = tiny_config([100003, 4096, 17], 8, opt=configs.ADAM, grad_dtype=configs.BF16)
+        pair = Pair(cfg)
+        try:
+            for it in range(2):
+                pair.push_iteration(it)
+                pair.aggregate(configs.rounds_all(cfg)[0])
+            outs.append([pair.gpu_block(0, b)[:3] for b in range(3)] + [pair.svc.block_stats(0, 0)])
+        finally:
+            pair.close()
+    for x, y in zip(outs[0][:3], outs[1][:3]):
+        for a, b in zip(x, y):
+            assert np.array_equal(a, b)
+    assert outs[0][3] == outs[1][3]      # the norm is reduced in a fixed order
+
+
+def test_bsp_bookkeeping_and_errors_on_device():
+    cfg = tiny_config([1000, 2000], 2)
+    pair = Pair(cfg)
+    svc = pair.svc
+    try:
+        g = torch.zeros(2000, device="cuda")
+        svc.push(0, 0, 0, g)
+        with pytest.raises(B.PsError) as e:
+            svc.aggregate([(0, 0)])
+        assert e.value.status == B.PS_ERR_NOT_READY
+        with pytest.raises(B.PsError) as e:
+            svc.push(0, 0, 0, g)
+        assert e.value.status == B.PS_ERR_DUPLICATE
+        svc.push(0, 0, 1, g)
+        with pytest.raises(B.PsError) as e:
+            svc.aggregate([(0, 0), (0, 0)])
+        assert e.value.status == B.PS_ERR_DUPLICATE
+        with pytest.raises(B.PsError) as e:
+            svc.aggregate([(0, 0), (0, 1)])
+        assert e.value.status == B.PS_ERR_NOT_READY
+        assert svc.block_stats(0, 0) == (0.0, 0)
+        before = svc.launch_info()["launches"]
+        svc.aggregate([])
+        assert svc.launch_info()["launches"] == before
+        svc.aggregate([(0, 0)])
+        assert svc.block_stats(0, 0) == (0.0, 1)
+        assert svc.launch_info()["launches"] == before + 1
+        with pytest.raises(B.PsError) as e:
+            svc.aggregate([(0, 0)])          # pushes were consumed
+        assert e.value.status == B.PS_ERR_NOT_READY
+    finally:
+        pair.close()
+
+
+def test_sqnorm_all_ones_and_host_push_pull():
+    cfg = tiny_config([50000], 2, lr=0.5, momentum=0.0, weight_decay=0.0)
+    pair = Pair(cfg)
+    svc = pair.svc
+    try:
+        ones = torch.ones(50000).pin_memory()
+        s = torch.cuda.Stream()
+        svc.push_host(0, 0, 0, ones, s)
+        svc.push_host(0, 0, 1, ones, s)
+        svc.aggregate([(0, 0)], s)
+        out = torch.empty(50000).pin_memory()
+        svc.pull_host(0, 0, out, s)
+        s.synchronize()
+        sq, step = svc.block_stats(0, 0)
+        assert sq == 4.0 * 50000 and step == 1
+        p0 = generate.init_params(cfg, 0)
+        assert torch.equal(out, p0 - 0.5 * 2.0)
+    finally:
+        pair.close()
