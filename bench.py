@@ -123,7 +123,7 @@ class Workload:
         from paper_2204_03211_b200 import binding as B
         self.B, self.cfg, self.device = B, cfg, device
         dev = torch.device("cuda", device)
-        arena = sum(3 * (4 * b.nelem + 256) for j in cfg.jobs for b in j.blocks) // cfg.num_contexts + (64 << 20)
+        arena = sum(3 * (4 * b.nelem + 256) for j in cfg.jobs for b in j.blocks) + (64 << 20)
         self.svc = B.Service(device, cfg.num_contexts, arena)
         self.slabs = []
         for j, job in enumerate(cfg.jobs):
@@ -149,7 +149,7 @@ class Workload:
                     for w in range(job.num_workers):
                         jobs.append(j); blocks.append(b); workers.append(w)
                         ptrs.append(base + (w * job.num_params + blk.job_offset) * esz)
-                rounds.append(dict(ready=ready, tasks=B.make_tasks(ready),
+                rounds.append(dict(ready=ready, tasks=B.make_tasks(ready), pulled=np.empty(len(ready), np.uint64),
                                    jobs=np.array(jobs, np.int32), blocks=np.array(blocks, np.int32),
                                    workers=np.array(workers, np.int32), ptrs=np.array(ptrs, np.uint64)))
             self.schedules.append(rounds)
@@ -163,8 +163,7 @@ class Workload:
         for r in rounds:
             svc.push_batch(r["jobs"], r["blocks"], r["workers"], r["ptrs"])
             svc.aggregate(r["tasks"], stream)
-            for (j, b) in r["ready"]:
-                svc.pull(j, b)
+            svc.pull_batch(r["tasks"], r["pulled"])
         return len(rounds)
 
     # ---- end to end: host gradients in, host parameters out
@@ -390,7 +389,7 @@ def main():
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         items, params, desc = oracle_sample(cfg, wl.slabs)
-        v, used, passes, el = time_oracle(items, params, 10.0, 50)
+        v, used, passes, el = time_oracle(items, params, 12.0, 1000)
         cpu = {"value": v, "unit": UNIT, "cores": used, "kind": "oracle",
                "sample": "%s, %d passes in %.1f s" % (desc, passes, el)}
 

@@ -78,7 +78,9 @@ enum {
                               Must be a multiple of 1024 (<= 2^20) when non-zero. */
   PS_OPT_CTAS_PER_SM = 2,  /* persistent CTAs per SM; 0 = automatic */
   PS_OPT_SORT_TASKS = 3,   /* 1 (default): heaviest chunks first inside a launch; 0: caller's order */
-  PS_OPT_KERNEL = 4        /* kernel variant: 0 = automatic; see ps_kernel_name */
+  PS_OPT_KERNEL = 4        /* kernel variant: 0 = automatic (bulk-copy ring), 1 = direct loads,
+                              2 = bulk-copy ring; results are identical except for the
+                              rounding of the per-block norm */
 };
 
 /* Creates an Aggregator service on GPU `device` with `num_contexts` contexts
@@ -151,6 +153,10 @@ int ps_aggregate(ps_service* svc, const ps_task* ready, int n_ready, void* strea
  * ps_migrate_block enqueued for the block has completed on its stream. */
 int ps_pull(ps_service* svc, int job, int block, const float** params_dev_ptr_out);
 
+/* Pull for n tasks in one call: out[i] receives the parameter pointer of
+ * tasks[i] (host arrays).  All-or-nothing. */
+int ps_pull_batch(ps_service* svc, const ps_task* tasks, int n, const float** params_dev_ptrs_out);
+
 /* Pull into host memory: enqueues a device-to-host copy of the parameters on
  * `stream` (ordered after the block's last aggregate/migration). */
 int ps_pull_host(ps_service* svc, int job, int block, float* params_host_dst, void* stream);
@@ -203,6 +209,11 @@ int ps_arena_info(ps_service* svc, int ctx, size_t* used_out, size_t* largest_fr
  * variant name of the last one (for launch accounting in benchmarks). */
 int ps_launch_info(ps_service* svc, unsigned long long* launches_out, int* grid_out, int* block_out,
                    const char** kernel_name_out);
+
+/* Waits for the device and reports the kernels' status word: 0 = no fault;
+ * non-zero = a bounded wait inside a kernel expired (the launch returned early
+ * and its results are undefined). */
+int ps_device_status(ps_service* svc, int* status_out);
 
 const char* ps_strerror(int status);
 /* Text of the last CUDA error seen by this service ("" if none). */

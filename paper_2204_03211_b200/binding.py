@@ -58,6 +58,7 @@ _SIGNATURES = {
     "ps_push_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
     "ps_aggregate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "ps_pull": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p)]),
+    "ps_pull_batch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "ps_pull_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
     "ps_migrate_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]),
     "ps_block_stats": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_ulonglong)]),
@@ -69,6 +70,7 @@ _SIGNATURES = {
     "ps_arena_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
     "ps_launch_info": (C.c_int, [C.c_void_p, C.POINTER(C.c_ulonglong), C.POINTER(C.c_int), C.POINTER(C.c_int),
                                  C.POINTER(C.c_char_p)]),
+    "ps_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int)]),
     "ps_strerror": (C.c_char_p, [C.c_int]),
     "ps_last_cuda_error": (C.c_char_p, [C.c_void_p]),
     "ps_version": (C.c_char_p, []),
@@ -179,6 +181,16 @@ def ps_pull(svc, job: int, block: int) -> int:
     return out.value
 
 
+def ps_pull_batch(svc, tasks, out=None):
+    """tasks: ctypes ps_task array (make_tasks); out: optional uint64 numpy
+    array to receive the pointers.  Returns the array of device pointers."""
+    import numpy as np
+    if out is None:
+        out = np.empty(len(tasks), np.uint64)
+    _check(load().ps_pull_batch(svc, tasks, len(tasks), out.ctypes.data), "ps_pull_batch", svc)
+    return out
+
+
 def ps_pull_host(svc, job: int, block: int, dst_host, stream=None):
     _check(load().ps_pull_host(svc, job, block, _ptr(dst_host), _stream_ptr(stream)), "ps_pull_host", svc)
 
@@ -228,6 +240,12 @@ def ps_launch_info(svc):
     n, g, b, name = C.c_ulonglong(), C.c_int(), C.c_int(), C.c_char_p()
     _check(load().ps_launch_info(svc, C.byref(n), C.byref(g), C.byref(b), C.byref(name)), "ps_launch_info", svc)
     return dict(launches=n.value, grid=g.value, block=b.value, kernel=(name.value or b"").decode())
+
+
+def ps_device_status(svc) -> int:
+    v = C.c_int()
+    _check(load().ps_device_status(svc, C.byref(v)), "ps_device_status", svc)
+    return v.value
 
 
 # ---- object wrapper -----------------------------------------------------------
@@ -280,7 +298,7 @@ def _bind(name):
     return method
 
 
-for _n in ("register_job", "register_block", "push", "push_batch", "push_host", "aggregate", "pull", "pull_host",
+for _n in ("register_job", "register_block", "push", "push_batch", "push_host", "aggregate", "pull", "pull_batch", "pull_host",
            "migrate_block", "block_stats", "block_state", "plan", "set_option", "get_option", "arena_info",
-           "launch_info"):
+           "launch_info", "device_status"):
     setattr(Service, _n, _bind(_n))

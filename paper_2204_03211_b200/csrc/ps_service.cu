@@ -106,6 +106,7 @@ struct ps_service {
   int next_slot = 0;
   unsigned long long gen = 0;              // ready-list generation
   long long opt_chunk = 0, opt_ctas = 0, opt_sort = 1, opt_kernel = 0;
+  int* status_dev = nullptr;               // error word written by kernels whose waits expired
   int occ_ctas = 0;
   unsigned long long launches = 0;
   int last_grid = 0, last_block = 0;
@@ -218,28 +219,40 @@ int validate_ready(ps_service* s, const ps_task* ready, int n_ready, std::vector
 
 size_t bytes_per_elem(const Job& j) { return (size_t)j.d.num_workers * j.grad_esize() + 8 * (1 + j.nstate()); }
 
-unsigned int pick_chunk_elems(ps_service* s, const std::vector<int>& idx, int grid_cap) {
+bool use_bulk(const ps_service* s) { return s->opt_kernel != 1; }
+
+int grid_cap(ps_service* s) {
+  int per_sm;
+  if (use_bulk(s)) per_sm = 1;   // one warp-specialised CTA owns an SM's shared memory
+  else per_sm = s->opt_ctas > 0 ? (int)s->opt_ctas : (s->occ_ctas > 0 ? s->occ_ctas : 3);
+  return s->num_sms * per_sm;
+}
+
+unsigned int pick_chunk_elems(ps_service* s, const std::vector<int>& idx) {
   if (s->opt_chunk > 0) return (unsigned int)s->opt_chunk;
   // Aim for ~16 chunks per resident CTA so that the tail of a launch is short,
-  // within [1024, 4096] elements.
+  // within [2048, 8192] elements.
   unsigned long long total = 0;
   for (int bi : idx) total += s->blocks[bi].nelem;
-  unsigned long long want = total / ((unsigned long long)grid_cap * 16ull);
-  unsigned int c = 4096;
-  while (c > 1024 && c > want) c >>= 1;
+  unsigned long long want = total / ((unsigned long long)grid_cap(s) * 16ull);
+  unsigned int c = 8192;
+  while (c > 2048 && c > want) c >>= 1;
   return c;
 }
 
-int grid_cap(ps_service* s) {
-  const int per_sm = s->opt_ctas > 0 ? (int)s->opt_ctas : (s->occ_ctas > 0 ? s->occ_ctas : 3);
-  return s->num_sms * per_sm;
+// Elements per ring tile of the bulk-copy kernel: the largest multiple of 128
+// whose rows (W shards, parameters, state) fit one stage; 0 if none does.
+unsigned int tile_elems_for(const Job& j) {
+  const size_t in_bytes = (size_t)j.d.num_workers * j.grad_esize() + 4 * (1 + j.nstate());
+  const size_t t = (size_t)kStageBytes / in_bytes / kTileQuantum * kTileQuantum;
+  return (unsigned int)t;
 }
 
 // Builds the task table for the validated blocks `idx`.
 int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
   const size_t n = idx.size();
   plan->order = idx;
-  plan->chunk_elems = pick_chunk_elems(s, idx, grid_cap(s));
+  plan->chunk_elems = pick_chunk_elems(s, idx);
   const unsigned int ce = plan->chunk_elems;
   if (s->opt_sort) {
     // heaviest chunks first: the launch's tail is then made of light chunks
@@ -287,6 +300,7 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
       if (reinterpret_cast<uintptr_t>(b.pushed[w]) & 15u) vec = 0;
     }
     t.vec_ok = vec;
+    t.tile_elems = tile_elems_for(j);
     starts[i] = t.first_chunk;
     row += j.d.num_workers;
     chunk += t.nchunks;
@@ -301,6 +315,7 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
   h->tasks_off = (unsigned int)tasks_off;
   h->starts_off = (unsigned int)starts_off;
   h->ptrs_off = (unsigned int)ptrs_off;
+  h->parts_per_chunk = use_bulk(s) ? kBulkConsumerWarps : 1;
   return PS_OK;
 }
 
@@ -376,6 +391,10 @@ int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->num_sms, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess)
       e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&s->occ_ctas, ps_aggregate_ldg_kernel, kThreads, 0);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(ps_aggregate_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBulkSmemBytes);
+    if (e == cudaSuccess) e = cudaMalloc(&s->status_dev, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(s->status_dev, 0, sizeof(int));
     for (int c = 0; e == cudaSuccess && c < num_contexts; ++c) {
       void* base = nullptr;
       e = cudaMalloc(&base, s->ctxs[c].arena.capacity() ? s->ctxs[c].arena.capacity() : Arena::kAlign);
@@ -384,6 +403,7 @@ int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes
     if (e != cudaSuccess) {
       const bool oom = (e == cudaErrorMemoryAllocation);
       for (auto& c : s->ctxs) if (c.base) cudaFree(c.base);
+      if (s->status_dev) cudaFree(s->status_dev);
       cudaGetLastError();
       delete s;
       return oom ? PS_ERR_NOMEM : PS_ERR_CUDA;
@@ -411,6 +431,7 @@ int ps_destroy(ps_service* s) {
     for (auto& c : s->ctxs) if (c.base) cudaFree(c.base);
     if (s->jobs_dev) cudaFree(s->jobs_dev);
     if (s->stats_dev) cudaFree(s->stats_dev);
+    if (s->status_dev) cudaFree(s->status_dev);
   }
   s->magic = 0;
   delete s;
@@ -555,7 +576,8 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
   rc = build_plan(s, idx, &plan);
   if (rc) return rc;
   Slot* sl = nullptr;
-  rc = acquire_slot(s, plan.bytes.size(), plan.total_chunks, &sl);
+  const bool bulk = use_bulk(s);
+  rc = acquire_slot(s, plan.bytes.size(), (size_t)plan.total_chunks * (bulk ? kBulkConsumerWarps : 1), &sl);
   if (rc) return rc;
   for (int bi : idx) {
     rc = order_after_block(s, s->blocks[bi], stream);
@@ -564,7 +586,11 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
   std::memcpy(sl->host, plan.bytes.data(), plan.bytes.size());
   PS_CUDA(s, cudaMemcpyAsync(sl->dev, sl->host, plan.bytes.size(), cudaMemcpyHostToDevice, stream));
   const int grid = (int)std::min<unsigned long long>(plan.total_chunks, (unsigned long long)grid_cap(s));
-  ps_aggregate_ldg_kernel<<<grid, kThreads, 0, stream>>>(sl->dev, s->jobs_dev, s->stats_dev, sl->partials);
+  if (bulk)
+    ps_aggregate_bulk_kernel<<<grid, kBulkThreads, kBulkSmemBytes, stream>>>(sl->dev, s->jobs_dev, s->stats_dev,
+                                                                             sl->partials, s->status_dev);
+  else
+    ps_aggregate_ldg_kernel<<<grid, kThreads, 0, stream>>>(sl->dev, s->jobs_dev, s->stats_dev, sl->partials);
   PS_CUDA(s, cudaGetLastError());
   PS_CUDA(s, cudaEventRecord(sl->done, stream));
   sl->inflight = true;
@@ -572,8 +598,8 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
   s->next_slot = (s->next_slot + 1) % kSlots;
   s->launches++;
   s->last_grid = grid;
-  s->last_block = kThreads;
-  s->last_kernel = "ldg";
+  s->last_block = bulk ? kBulkThreads : kThreads;
+  s->last_kernel = bulk ? "bulk" : "ldg";
   for (int bi : idx) {
     Block& b = s->blocks[bi];
     b.step++;
@@ -624,6 +650,17 @@ int ps_pull(ps_service* s, int job, int block, const float** out) {
   if (bi < 0 || !out) return PS_ERR_BAD_ARG;
   if (!has_device(s)) return PS_ERR_NO_DEVICE;
   *out = blk_p(s, s->blocks[bi]);
+  return PS_OK;
+}
+
+int ps_pull_batch(ps_service* s, const ps_task* tasks, int n, const float** out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (n < 0 || (n > 0 && (!tasks || !out))) return PS_ERR_BAD_ARG;
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  for (int i = 0; i < n; ++i)
+    if (find_block(s, tasks[i].job, tasks[i].block) < 0) return PS_ERR_BAD_ARG;
+  for (int i = 0; i < n; ++i) out[i] = blk_p(s, s->blocks[find_block(s, tasks[i].job, tasks[i].block)]);
   return PS_OK;
 }
 
@@ -733,7 +770,7 @@ int ps_set_option(ps_service* s, int option, long long value) {
       s->opt_sort = value ? 1 : 0;
       return PS_OK;
     case PS_OPT_KERNEL:
-      if (value < 0 || value > 1) return PS_ERR_BAD_ARG;
+      if (value < 0 || value > 2) return PS_ERR_BAD_ARG;
       s->opt_kernel = value;
       return PS_OK;
     default:
@@ -774,6 +811,18 @@ int ps_launch_info(ps_service* s, unsigned long long* launches, int* grid, int* 
   if (grid) *grid = s->last_grid;
   if (block) *block = s->last_block;
   if (name) *name = s->last_kernel;
+  return PS_OK;
+}
+
+int ps_device_status(ps_service* s, int* status_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (!status_out) return PS_ERR_BAD_ARG;
+  *status_out = 0;
+  if (!has_device(s)) return PS_OK;
+  PS_CUDA(s, cudaSetDevice(s->device));
+  PS_CUDA(s, cudaDeviceSynchronize());
+  PS_CUDA(s, cudaMemcpy(status_out, s->status_dev, sizeof(int), cudaMemcpyDeviceToHost));
   return PS_OK;
 }
 

@@ -35,11 +35,13 @@ def assert_close(got: np.ndarray, ref: np.ndarray, what: str, tol: float = TOL):
 class Pair:
     """One CUDA service and one oracle fed the same registrations and pushes."""
 
-    def __init__(self, cfg: configs.Config, device: int = 0, arena_bytes: int | None = None, nthreads: int = 0):
+    def __init__(self, cfg: configs.Config, device: int = 0, arena_bytes: int | None = None, nthreads: int = 0,
+                 kernel: int = 0):
         self.cfg = cfg
         self.dev = torch.device("cuda", device)
         need = sum(3 * (4 * b.nelem + 256) for j in cfg.jobs for b in j.blocks) + (1 << 20)
         self.svc = B.Service(device, cfg.num_contexts, arena_bytes or need)
+        self.svc.set_option(B.PS_OPT_KERNEL, kernel)
         self.ora = A.OracleAggregator(cfg.num_contexts, nthreads)
         self.keep = []          # gradient tensors of the iteration in flight
         for j, job in enumerate(cfg.jobs):
@@ -91,6 +93,7 @@ class Pair:
 
     def compare(self, sq_rtol: float = 1e-5, exact: bool = True):
         worst = 0.0
+        assert self.svc.device_status() == 0, "a bounded wait expired inside a kernel"
         for j, job in enumerate(self.cfg.jobs):
             for b in job.blocks:
                 p, a, v, ctx = self.gpu_block(j, b.block)

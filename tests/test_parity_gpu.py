@@ -14,10 +14,13 @@ ODD_SIZES = [1, 3, 4, 5, 127, 1024, 4097, 12289, 70001]
 
 @pytest.mark.parametrize("opt,dt", [(configs.SGD, configs.F32), (configs.ADAM, configs.F32),
                                     (configs.SGD, configs.BF16), (configs.ADAM, configs.BF16)])
-@pytest.mark.parametrize("W", [1, 2, 5, 8, 33])
-def test_odd_sizes_bit_exact(opt, dt, W):
+@pytest.mark.parametrize("W", [1, 2, 5, 8, 33, 70])
+@pytest.mark.parametrize("kernel", [1, 2], ids=["ldg", "bulk"])
+def test_odd_sizes_bit_exact(opt, dt, W, kernel):
+    # W = 70 with fp32 gradients exceeds what one ring stage can hold, so the
+    # bulk-copy kernel hands those chunks to its direct-load path.
     cfg = tiny_config(ODD_SIZES, W, opt=opt, grad_dtype=dt)
-    pair = Pair(cfg)
+    pair = Pair(cfg, kernel=kernel)
     try:
         every = configs.rounds_all(cfg)[0]
         for it in range(3):
@@ -29,9 +32,10 @@ def test_odd_sizes_bit_exact(opt, dt, W):
 
 
 @pytest.mark.parametrize("chunk", [1024, 2048, 8192, 65536])
-def test_chunk_size_and_order_invariance(chunk):
+@pytest.mark.parametrize("kernel", [1, 2], ids=["ldg", "bulk"])
+def test_chunk_size_and_order_invariance(chunk, kernel):
     cfg = tiny_config([5, 40000, 1024, 300001, 77], 4)
-    pair = Pair(cfg)
+    pair = Pair(cfg, kernel=kernel)
     try:
         pair.svc.set_option(B.PS_OPT_CHUNK_ELEMS, chunk)
         pair.svc.set_option(B.PS_OPT_SORT_TASKS, chunk % 2048 == 0)
@@ -44,9 +48,10 @@ def test_chunk_size_and_order_invariance(chunk):
         pair.close()
 
 
-def test_unaligned_shards_take_scalar_path_same_bits():
+@pytest.mark.parametrize("kernel", [1, 2], ids=["ldg", "bulk"])
+def test_unaligned_shards_take_scalar_path_same_bits(kernel):
     cfg = tiny_config([4099, 600], 3)
-    pair = Pair(cfg)
+    pair = Pair(cfg, kernel=kernel)
     try:
         job = cfg.jobs[0]
         slab = generate.grad_slab(cfg, 0, 0)
@@ -71,9 +76,10 @@ def test_unaligned_shards_take_scalar_path_same_bits():
         pair.close()
 
 
-def test_c1_ten_iterations():
+@pytest.mark.parametrize("kernel", [1, 2], ids=["ldg", "bulk"])
+def test_c1_ten_iterations(kernel):
     cfg = configs.c1()
-    pair = Pair(cfg)
+    pair = Pair(cfg, kernel=kernel)
     try:
         every = configs.rounds_all(cfg)[0]
         for it in range(cfg.iterations):
