@@ -148,7 +148,7 @@ class Workload:
                     base = self.slabs[j].data_ptr()
                     for w in range(job.num_workers):
                         jobs.append(j); blocks.append(b); workers.append(w)
-                        ptrs.append(base + (w * job.num_params + blk.job_offset) * esz)
+                        ptrs.append(generate.shard_ptr(self.slabs[j], w, blk.job_offset))
                 rounds.append(dict(ready=ready, tasks=B.make_tasks(ready), pulled=np.empty(len(ready), np.uint64),
                                    jobs=np.array(jobs, np.int32), blocks=np.array(blocks, np.int32),
                                    workers=np.array(workers, np.int32), ptrs=np.array(ptrs, np.uint64)))
@@ -176,7 +176,7 @@ class Workload:
         flat = self.pool.view(torch.uint8)
         off = 0
         for s in self.slabs:
-            src = s.view(-1).view(torch.uint8)
+            src = (s._base if s._base is not None else s).view(-1).view(torch.uint8)
             n = min(src.numel(), flat.numel() - off)
             if n <= 0:
                 break

@@ -65,13 +65,13 @@ class Pair:
             if jobs is not None and j not in jobs:
                 continue
             slab = generate.grad_slab(self.cfg, j, it)
-            dslab = slab.to(self.dev)
+            dslab = generate.to_device(slab, self.dev)
             self.keep.append((slab, dslab))
             host = to_np(slab)
             esz = dslab.element_size()
             for b in job.blocks:
                 for w in range(job.num_workers):
-                    self.svc.push(j, b.block, w, dslab.data_ptr() + (w * job.num_params + b.job_offset) * esz)
+                    self.svc.push(j, b.block, w, generate.shard_ptr(dslab, w, b.job_offset))
                     self.ora.push(j, b.block, w, host[w, b.job_offset:b.job_offset + b.nelem])
 
     def aggregate(self, ready, stream=None):

@@ -15,6 +15,27 @@ import torch
 from .configs import BF16, Config, JobSpec
 
 
+ROW_ALIGN_ELEMS = 128   # shard rows start at multiples of 128 elements (256 B for bf16, 512 B for fp32)
+
+
+def shard_ptr(slab: torch.Tensor, worker: int, elem_offset: int) -> int:
+    """Device/host address of element `elem_offset` of worker `worker`'s shard."""
+    return slab.data_ptr() + (worker * slab.stride(0) + elem_offset) * slab.element_size()
+
+
+def empty_slab(W: int, P: int, dtype, device) -> torch.Tensor:
+    """[W, P] view whose rows start on ROW_ALIGN_ELEMS boundaries of one buffer."""
+    pad = (P + ROW_ALIGN_ELEMS - 1) // ROW_ALIGN_ELEMS * ROW_ALIGN_ELEMS
+    return torch.empty((W, pad), dtype=dtype, device=device)[:, :P]
+
+
+def to_device(slab: torch.Tensor, device) -> torch.Tensor:
+    """Copy of a slab on `device` with the same padded row layout."""
+    out = empty_slab(slab.shape[0], slab.shape[1], slab.dtype, device)
+    out.copy_(slab)
+    return out
+
+
 def _seed(*key) -> int:
     return int(np.random.SeedSequence(list(key)).generate_state(1, dtype=np.uint64)[0] >> 1)
 
@@ -54,7 +75,9 @@ def grad_slab(cfg: Config, job: int, iteration: int, device="cpu", out: torch.Te
     W, P = spec.num_workers, spec.num_params
     dt = torch.bfloat16 if spec.grad_dtype == BF16 else torch.float32
     if out is None:
-        out = torch.empty((W, P), dtype=dt, device=device)
+        # every worker's shard starts on a 256-byte boundary, as separately
+        # allocated gradient buffers would: rows are padded, the view is [W, P]
+        out = empty_slab(W, P, dt, device)
     assert out.shape == (W, P) and out.dtype == dt
     gen = _gen(out.device, cfg.seed, 13, job, iteration)
     full = torch.empty((W, P), dtype=torch.float32, device=out.device) if keep_fp32 else None
