@@ -57,7 +57,8 @@ typedef enum {
   PS_ERR_ALIGN = -5,      /* gradient pointer not aligned to its element size */
   PS_ERR_NOMEM = -6,      /* context arena (or host/device allocation) exhausted */
   PS_ERR_CUDA = -7,       /* a CUDA runtime call failed; see ps_last_cuda_error */
-  PS_ERR_NO_DEVICE = -8   /* service was created without a device (planning only) */
+  PS_ERR_NO_DEVICE = -8,  /* service was created without a device (planning only) */
+  PS_ERR_TOO_LARGE = -9   /* ps_aggregate_block_noalloc: nelem above PS_NOALLOC_MAX_ELEMS */
 } ps_status;
 
 typedef struct {
@@ -214,6 +215,41 @@ int ps_launch_info(ps_service* svc, unsigned long long* launches_out, int* grid_
  * non-zero = a bounded wait inside a kernel expired (the launch returned early
  * and its results are undefined). */
 int ps_device_status(ps_service* svc, int* status_out);
+
+/* Largest block ps_aggregate_block_noalloc accepts (2^24 elements). */
+#define PS_NOALLOC_MAX_ELEMS ((size_t)1 << 24)
+
+/* Aggregates ONE block without allocating anything, for callers that must not
+ * touch the allocator.  (The paper has no counterpart: this is a convenience of
+ * this library.)  Typical callers: a process whose framework has already
+ * reserved all device memory for its own pool, so a cudaMalloc here could fail
+ * or fragment it; a latency-critical loop that cannot take the implicit
+ * device-wide synchronisation an allocation may cause; code that runs where the
+ * memory budget is fixed at start-up.  No ps_service is involved: the caller
+ * owns and passes everything —
+ *   job                hyper-parameters (host pointer; W = job->num_workers)
+ *   step               t >= 1, the number of this aggregate for the block
+ *   nelem              1 .. PS_NOALLOC_MAX_ELEMS, else PS_ERR_TOO_LARGE
+ *   params/state0/state1   device pointers to nelem floats, updated in place
+ *                      (state1 = Adam's second moment, NULL for SGD)
+ *   shard_dev_ptrs     host array of W device pointers to the gradient shards
+ *   sqnorm_dev_out     device pointer that receives sum G*G, or NULL
+ * and gets the same arithmetic as ps_aggregate (same kernel).  The work is
+ * enqueued on `stream` of the CURRENT device; nothing is waited for.
+ *
+ * The kernel's scratch (task table, work counter, per-chunk partial sums: 20 KB)
+ * lives in a fixed array inside the library's device image, so every GPU that
+ * loads the library holds those 20 KB until the process exits.  The first call
+ * on a device looks the array's address up and caches it; make that first call
+ * outside any stream capture.  All calls on a device share the array and each
+ * call re-initialises the parts that must start at zero, so calls must not
+ * overlap on the GPU: issue them on one stream, or order the streams yourself.
+ * Calls cudaMalloc/cudaFree never.  Errors: BAD_ARG, ALIGN (a pointer not
+ * 4-byte / element aligned), TOO_LARGE, CUDA. */
+int ps_aggregate_block_noalloc(const ps_job_desc* job, unsigned long long step, size_t nelem,
+                               float* params_dev, float* state0_dev, float* state1_dev_or_null,
+                               const void* const* shard_dev_ptrs, double* sqnorm_dev_out_or_null,
+                               void* stream);
 
 const char* ps_strerror(int status);
 /* Text of the last CUDA error seen by this service ("" if none). */

@@ -19,6 +19,8 @@ PS_F32, PS_BF16 = 0, 1
 PS_OK = 0
 PS_ERR_BAD_HANDLE, PS_ERR_BAD_ARG, PS_ERR_DUPLICATE, PS_ERR_NOT_READY = -1, -2, -3, -4
 PS_ERR_ALIGN, PS_ERR_NOMEM, PS_ERR_CUDA, PS_ERR_NO_DEVICE = -5, -6, -7, -8
+PS_ERR_TOO_LARGE = -9
+PS_NOALLOC_MAX_ELEMS = 1 << 24
 PS_DEVICE_NONE = -1
 PS_MAX_WORKERS = 256
 PS_OPT_CHUNK_ELEMS, PS_OPT_CTAS_PER_SM, PS_OPT_SORT_TASKS, PS_OPT_KERNEL = 1, 2, 3, 4
@@ -71,6 +73,8 @@ _SIGNATURES = {
     "ps_launch_info": (C.c_int, [C.c_void_p, C.POINTER(C.c_ulonglong), C.POINTER(C.c_int), C.POINTER(C.c_int),
                                  C.POINTER(C.c_char_p)]),
     "ps_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int)]),
+    "ps_aggregate_block_noalloc": (C.c_int, [C.POINTER(ps_job_desc), C.c_ulonglong, C.c_size_t, C.c_void_p,
+                                             C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ps_strerror": (C.c_char_p, [C.c_int]),
     "ps_last_cuda_error": (C.c_char_p, [C.c_void_p]),
     "ps_version": (C.c_char_p, []),
@@ -240,6 +244,17 @@ def ps_launch_info(svc):
     n, g, b, name = C.c_ulonglong(), C.c_int(), C.c_int(), C.c_char_p()
     _check(load().ps_launch_info(svc, C.byref(n), C.byref(g), C.byref(b), C.byref(name)), "ps_launch_info", svc)
     return dict(launches=n.value, grid=g.value, block=b.value, kernel=(name.value or b"").decode())
+
+
+def ps_aggregate_block_noalloc(job_desc: ps_job_desc, step: int, nelem: int, params, state0, state1, shards,
+                               sqnorm_out=None, stream=None):
+    """One block through the entry point that allocates nothing (see the
+    header).  params/state0/state1/sqnorm_out: device tensors or addresses;
+    shards: list of W device tensors or addresses."""
+    arr = (C.c_void_p * len(shards))(*[_ptr(g) for g in shards])
+    _check(load().ps_aggregate_block_noalloc(C.byref(job_desc), step, nelem, _ptr(params), _ptr(state0),
+                                             _ptr(state1), arr, _ptr(sqnorm_out), _stream_ptr(stream)),
+           "ps_aggregate_block_noalloc")
 
 
 def ps_device_status(svc) -> int:

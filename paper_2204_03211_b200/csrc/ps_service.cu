@@ -839,6 +839,7 @@ const char* ps_strerror(int status) {
     case PS_ERR_NOMEM: return "out of arena, device or host memory";
     case PS_ERR_CUDA: return "CUDA runtime error";
     case PS_ERR_NO_DEVICE: return "service has no device (planning only)";
+    case PS_ERR_TOO_LARGE: return "block larger than PS_NOALLOC_MAX_ELEMS";
     default: return "unknown status";
   }
 }
@@ -848,3 +849,152 @@ const char* ps_last_cuda_error(ps_service* s) { return alive(s) ? s->cuda_err.c_
 const char* ps_version(void) { return "ps_b200 0.1 (sm_100a)"; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// ps_aggregate_block_noalloc: one block, no allocation of any kind.
+//
+// The aggregation kernel needs a little global memory besides its inputs and
+// outputs: the task table it walks, the work counter, one partial sum per chunk
+// and the statistics record.  Here that scratch is a fixed array in the
+// library's device image.  In host code the array's name is only a handle for
+// the runtime, not a device address: the address comes from
+// cudaGetSymbolAddress, once per device with that device current, and is what
+// the kernels are given.  Device code (the two small kernels below) names the
+// array directly.
+// ---------------------------------------------------------------------------
+namespace psb {
+
+constexpr unsigned int kNaChunk = 8192;                                   // elements per chunk
+constexpr size_t kNaMaxChunks = PS_NOALLOC_MAX_ELEMS / kNaChunk;          // 2048
+constexpr size_t kNaTaskOff = sizeof(PsTableHdr);                         // 32
+constexpr size_t kNaStartsOff = kNaTaskOff + sizeof(PsTaskDev);           // 112
+constexpr size_t kNaPtrsOff = 128;
+constexpr size_t kNaJobOff = kNaPtrsOff + PS_MAX_WORKERS * sizeof(void*); // 2176
+constexpr size_t kNaStatOff = kNaJobOff + sizeof(PsJobDev);               // 2240
+constexpr size_t kNaPartOff = 2304;
+constexpr size_t kNaScratchBytes = kNaPartOff + kNaMaxChunks * sizeof(double);   // 18688
+static_assert(kNaStartsOff + sizeof(unsigned int) <= kNaPtrsOff, "scratch layout");
+static_assert(kNaStatOff + sizeof(PsStat) <= kNaPartOff, "scratch layout");
+static_assert(kNaScratchBytes <= 20480, "scratch stays at 20 KB");
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[20480];
+
+struct NoAllocArgs {            // passed by value as kernel parameters (< 4 KB)
+  PsJobDev job;
+  PsTaskDev task;
+  const void* shards[PS_MAX_WORKERS];
+};
+
+// Writes this call's task table into the scratch array; everything that must
+// start at zero (work counter, ticket, statistics) is rewritten on every call
+// because the array keeps the previous call's contents.
+__global__ void ps_noalloc_setup_kernel(NoAllocArgs a) {
+  unsigned char* base = g_noalloc_scratch;
+  const unsigned int t = threadIdx.x;
+  if (t < (unsigned int)a.job.W) reinterpret_cast<const void**>(base + kNaPtrsOff)[t] = a.shards[t];
+  if (t == 0) {
+    PsTableHdr h;
+    h.counter = 0;
+    h.n_tasks = 1;
+    h.total_chunks = a.task.nchunks;
+    h.chunk_elems = kNaChunk;
+    h.tasks_off = (unsigned int)kNaTaskOff;
+    h.starts_off = (unsigned int)kNaStartsOff;
+    h.ptrs_off = (unsigned int)kNaPtrsOff;
+    h.parts_per_chunk = 1;
+    *reinterpret_cast<PsTableHdr*>(base) = h;
+    *reinterpret_cast<PsTaskDev*>(base + kNaTaskOff) = a.task;     // ticket = 0 inside
+    *reinterpret_cast<unsigned int*>(base + kNaStartsOff) = 0;
+    *reinterpret_cast<PsJobDev*>(base + kNaJobOff) = a.job;
+    PsStat z;
+    z.sqnorm = 0.0;
+    z.step = 0;
+    *reinterpret_cast<PsStat*>(base + kNaStatOff) = z;
+  }
+}
+
+__global__ void ps_noalloc_finish_kernel(double* out) {
+  *out = reinterpret_cast<const PsStat*>(g_noalloc_scratch + kNaStatOff)->sqnorm;
+}
+
+struct NoAllocDevice {
+  unsigned char* scratch = nullptr;   // device address of g_noalloc_scratch on this device
+  int num_sms = 0;
+};
+constexpr int kNaMaxDevices = 64;
+static NoAllocDevice g_na_dev[kNaMaxDevices];
+static std::mutex g_na_mu;
+
+}  // namespace psb
+
+extern "C" int ps_aggregate_block_noalloc(const ps_job_desc* job, unsigned long long step, size_t nelem,
+                                          float* params, float* state0, float* state1,
+                                          const void* const* shard_ptrs, double* sqnorm_out, void* stream_) {
+  if (!job || !params || !state0 || !shard_ptrs || step < 1 || nelem == 0) return PS_ERR_BAD_ARG;
+  if (job->opt != PS_SGD && job->opt != PS_ADAM) return PS_ERR_BAD_ARG;
+  if (job->grad_dtype != PS_F32 && job->grad_dtype != PS_BF16) return PS_ERR_BAD_ARG;
+  if (job->num_workers < 1 || job->num_workers > PS_MAX_WORKERS) return PS_ERR_BAD_ARG;
+  if (job->opt == PS_ADAM && !state1) return PS_ERR_BAD_ARG;
+  if (nelem > PS_NOALLOC_MAX_ELEMS) return PS_ERR_TOO_LARGE;
+  const uintptr_t esz = job->grad_dtype == PS_BF16 ? 2 : 4;
+  uintptr_t all = reinterpret_cast<uintptr_t>(params) | reinterpret_cast<uintptr_t>(state0) |
+                  reinterpret_cast<uintptr_t>(state1) | reinterpret_cast<uintptr_t>(sqnorm_out);
+  if ((all & 3u) || (reinterpret_cast<uintptr_t>(sqnorm_out) & 7u)) return PS_ERR_ALIGN;
+  for (int w = 0; w < job->num_workers; ++w) {
+    if (!shard_ptrs[w]) return PS_ERR_BAD_ARG;
+    if (reinterpret_cast<uintptr_t>(shard_ptrs[w]) & (esz - 1)) return PS_ERR_ALIGN;
+    all |= reinterpret_cast<uintptr_t>(shard_ptrs[w]);
+  }
+
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNaMaxDevices) return PS_ERR_CUDA;
+  NoAllocDevice nd;
+  {
+    // first call on this device: look the scratch array's address up (the
+    // device is current, as the runtime requires) and remember it
+    std::lock_guard<std::mutex> lk(g_na_mu);
+    if (!g_na_dev[dev].scratch) {
+      void* ptr = nullptr;
+      if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return PS_ERR_CUDA;
+      int sms = 0;
+      if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        return PS_ERR_CUDA;
+      g_na_dev[dev].num_sms = sms;
+      g_na_dev[dev].scratch = static_cast<unsigned char*>(ptr);
+    }
+    nd = g_na_dev[dev];
+  }
+
+  NoAllocArgs a;
+  std::memset(&a, 0, sizeof a);
+  a.job.opt = job->opt; a.job.grad_dtype = job->grad_dtype; a.job.W = job->num_workers;
+  a.job.lr = job->lr; a.job.mom = job->momentum; a.job.wd = job->weight_decay;
+  a.job.b1 = job->beta1; a.job.b2 = job->beta2;
+  a.job.omb1 = 1.0f - job->beta1;
+  a.job.omb2 = 1.0f - job->beta2;
+  a.job.eps = job->eps; a.job.gs = job->grad_scale;
+  a.task.p = params; a.task.s0 = state0; a.task.s1 = state1;
+  a.task.nelem = nelem;
+  a.task.shard_row = 0;
+  a.task.first_chunk = 0;
+  a.task.nchunks = (unsigned int)((nelem + kNaChunk - 1) / kNaChunk);
+  a.task.ticket = 0;
+  a.task.ss_t = (float)((double)job->lr / (1.0 - std::pow((double)job->beta1, (double)step)));
+  a.task.sbc2_t = (float)std::sqrt(1.0 - std::pow((double)job->beta2, (double)step));
+  a.task.job = 0;
+  a.task.stat_idx = 0;
+  a.task.step = step;
+  a.task.vec_ok = (all & 15u) ? 0u : 1u;
+  a.task.tile_elems = 0;
+  for (int w = 0; w < job->num_workers; ++w) a.shards[w] = shard_ptrs[w];
+
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  unsigned char* sc = nd.scratch;
+  ps_noalloc_setup_kernel<<<1, PS_MAX_WORKERS, 0, stream>>>(a);
+  const int grid = (int)std::min<unsigned long long>(a.task.nchunks, (unsigned long long)nd.num_sms * 3ull);
+  ps_aggregate_ldg_kernel<<<grid, kThreads, 0, stream>>>(sc, reinterpret_cast<const PsJobDev*>(sc + kNaJobOff),
+                                                         reinterpret_cast<PsStat*>(sc + kNaStatOff),
+                                                         reinterpret_cast<double*>(sc + kNaPartOff));
+  if (sqnorm_out) ps_noalloc_finish_kernel<<<1, 1, 0, stream>>>(sqnorm_out);
+  return cudaGetLastError() == cudaSuccess ? PS_OK : PS_ERR_CUDA;
+}
