@@ -306,6 +306,7 @@ def main():
     ap.add_argument("--ticks", type=int, default=16, help="rounds per iteration window of the arrival schedule")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--host-pool-gb", type=float, default=8.0)
+    ap.add_argument("--jobs", default="", help="comma-separated subset of the workload's jobs (profiling a small case)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -315,6 +316,9 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     cfg = configs.CONFIGS[args.workload]()
+    if args.jobs:
+        cfg.jobs = [cfg.jobs[int(x)] for x in args.jobs.split(",")]
+        cfg.name += "[jobs %s]" % args.jobs
     config = {"workload": "%s: %d packed jobs, %d params, %d blocks, W=%s, %s arrival in <=%d rounds/step" % (
         cfg.name, len(cfg.jobs), cfg.num_params, sum(len(j.blocks) for j in cfg.jobs),
         sorted({j.num_workers for j in cfg.jobs}), cfg.arrival, args.ticks),
