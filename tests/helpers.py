@@ -128,3 +128,130 @@ def tiny_config(sizes, W, opt=configs.SGD, grad_dtype=configs.F32, seed=123, **k
     base.update(kw)
     job = configs.JobSpec("tiny", "tiny", tensors, blocks, W, opt=opt, grad_dtype=grad_dtype, **base)
     return configs.Config("tiny", seed, 3, [job])
+
+
+class SampledPair:
+    """Full-size configurations: the CUDA service holds every block; the oracle
+    follows (a) a seeded sample of positions of EVERY block (block edges, chunk
+    boundaries, random interior points) packed into one pseudo-block per job —
+    valid because the update is element-wise — and (b) a few whole blocks per
+    job, for which the per-block norm is checked too.  Gradients are generated
+    on the GPU; the oracle receives copies of exactly those bits."""
+
+    def __init__(self, cfg: configs.Config, per_block: int = 48, full_per_job: int = 4, device: int = 0,
+                 full_block_limit: int = 1 << 21):
+        self.cfg = cfg
+        self.dev = torch.device("cuda", device)
+        arena = sum(3 * (4 * b.nelem + 256) for j in cfg.jobs for b in j.blocks) + (64 << 20)
+        self.svc = B.Service(device, cfg.num_contexts, arena)
+        self.ora = A.OracleAggregator(1, 0)
+        self.pos, self.full = [], []
+        self.ctx = {}
+        for j, job in enumerate(cfg.jobs):
+            assert self.svc.register_job(**job.hparams()) == j == self.ora.register_job(oracle_hp(job))
+            p0 = generate.init_params(cfg, j, self.dev)
+            for b in job.blocks:
+                c = configs.initial_context(cfg, j, b.block)
+                self.ctx[(j, b.block)] = c
+                self.svc.register_block(j, b.block, b.nelem, c, p0[b.job_offset:b.job_offset + b.nelem])
+            pos = generate.sample_positions(cfg, j, per_block).to(self.dev)
+            self.pos.append(pos)
+            self.ora.register_block(j, 0, pos.numel(), 0, p0[pos].cpu().numpy())
+            # whole blocks: first, last, the smallest and the largest that is not huge
+            cand = [b for b in job.blocks if b.nelem <= full_block_limit]
+            pick = {cand[0].block, cand[-1].block, min(cand, key=lambda b: b.nelem).block,
+                    max(cand, key=lambda b: b.nelem).block}
+            pick = sorted(pick)[:full_per_job]
+            self.full.append(pick)
+            for k, bid in enumerate(pick):
+                b = job.blocks[bid]
+                self.ora.register_block(j, 1 + k, b.nelem, 0, p0[b.job_offset:b.job_offset + b.nelem].cpu().numpy())
+            del p0
+        self.slabs = [None] * len(cfg.jobs)
+
+    def close(self):
+        self.svc.close()
+
+    def iteration(self, it: int, rounds, stream=None):
+        """Pushes fresh gradients for every block, aggregates round by round."""
+        cfg = self.cfg
+        for j, job in enumerate(cfg.jobs):
+            self.slabs[j] = generate.grad_slab(cfg, j, it, self.dev, out=self.slabs[j])
+        torch.cuda.synchronize(self.dev)
+        for ready in rounds:
+            jobs, blocks, workers, ptrs = [], [], [], []
+            for (j, b) in ready:
+                job = cfg.jobs[j]
+                for w in range(job.num_workers):
+                    jobs.append(j); blocks.append(b); workers.append(w)
+                    ptrs.append(generate.shard_ptr(self.slabs[j], w, job.blocks[b].job_offset))
+            self.svc.push_batch(np.array(jobs, np.int32), np.array(blocks, np.int32), np.array(workers, np.int32),
+                                np.array(ptrs, np.uint64))
+            self.svc.aggregate(ready, stream)
+        # oracle: the same bits, sampled columns and whole blocks
+        for j, job in enumerate(cfg.jobs):
+            samp = to_np(self.slabs[j][:, self.pos[j]])
+            ready = [(j, 0)]
+            for w in range(job.num_workers):
+                self.ora.push(j, 0, w, samp[w])
+            for k, bid in enumerate(self.full[j]):
+                b = job.blocks[bid]
+                whole = to_np(self.slabs[j][:, b.job_offset:b.job_offset + b.nelem])
+                for w in range(job.num_workers):
+                    self.ora.push(j, 1 + k, w, whole[w])
+                ready.append((j, 1 + k))
+            self.ora.aggregate(ready)
+        torch.cuda.synchronize(self.dev)
+
+    def migrate(self, plan, stream=None):
+        for (j, b) in plan:
+            dst = (self.ctx[(j, b)] + 1) % self.cfg.num_contexts
+            self.svc.migrate_block(j, b, dst, stream)
+            self.ctx[(j, b)] = dst
+
+    def _gather(self, j: int):
+        """p, s0, s1 of job j at the sampled positions, from the service's memory."""
+        job = self.cfg.jobs[j]
+        pos = self.pos[j]
+        starts = torch.tensor([b.job_offset for b in job.blocks] + [job.num_params], device=self.dev)
+        which = torch.searchsorted(starts, pos, right=True) - 1
+        outs = [torch.empty(pos.numel(), device=self.dev) for _ in range(3)]
+        has_s1 = False
+        for b in job.blocks:
+            sel = (which == b.block).nonzero().squeeze(1)
+            if sel.numel() == 0:
+                continue
+            loc = pos[sel] - b.job_offset
+            s0, s1, ctx = self.svc.block_state(j, b.block)
+            assert ctx == self.ctx[(j, b.block)], "block (%d,%d) in the wrong context" % (j, b.block)
+            outs[0][sel] = self.svc.view(self.svc.pull(j, b.block), b.nelem)[loc]
+            outs[1][sel] = self.svc.view(s0, b.nelem)[loc]
+            if s1:
+                has_s1 = True
+                outs[2][sel] = self.svc.view(s1, b.nelem)[loc]
+        return outs[0].cpu().numpy(), outs[1].cpu().numpy(), outs[2].cpu().numpy() if has_s1 else None
+
+    def compare(self, expect_step: int, sq_rtol: float = 1e-5):
+        assert self.svc.device_status() == 0
+        torch.cuda.synchronize(self.dev)
+        for j, job in enumerate(self.cfg.jobs):
+            tag = "%s job %d" % (self.cfg.name, j)
+            p, a, v = self._gather(j)
+            rp = self.ora.pull(j, 0)
+            ra, rv = self.ora.state(j, 0)
+            assert_close(p, rp, tag + " sampled params")
+            assert_close(a, ra, tag + " sampled state0")
+            assert np.array_equal(p, rp) and np.array_equal(a, ra), tag + " samples not bit-identical"
+            if rv is not None:
+                assert_close(v, rv, tag + " sampled state1")
+                assert np.array_equal(v, rv), tag + " sampled state1 not bit-identical"
+            for k, bid in enumerate(self.full[j]):
+                n = job.blocks[bid].nelem
+                got = self.svc.view(self.svc.pull(j, bid), n).cpu().numpy()
+                assert np.array_equal(got, self.ora.pull(j, 1 + k)), tag + " whole block %d" % bid
+                sq, step = self.svc.block_stats(j, bid)
+                rsq, rstep = self.ora.block_stats(j, 1 + k)
+                assert step == rstep == expect_step, tag + " step of block %d" % bid
+                assert abs(sq - rsq) <= sq_rtol * abs(rsq) + 1e-300, tag + " sqnorm of block %d" % bid
+            for b in job.blocks[:: max(1, len(job.blocks) // 16)]:
+                assert self.svc.block_stats(j, b.block)[1] == expect_step
