@@ -214,6 +214,22 @@ class Workload:
         return len(rounds)
 
 
+def max_over_ranks(ms: float, device=None) -> float:
+    """Slowest rank's time (every rank gets it).  No-op without a process group."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank_per_step: int, world: int, steps: int, ms: float) -> float:
+    """Replicas only: every rank processes the same number of units; the job's
+    throughput is all ranks' units over the slowest rank's time."""
+    return world * units_per_rank_per_step * steps / (ms * 1e-3)
+
+
 def timed(fn, steps: int, stream, dist_on: bool, device):
     """Times `steps` calls of fn(k, stream) with CUDA events on `stream`,
     bracketed by barrier + synchronize; returns (ms max over ranks, launches)."""
@@ -233,11 +249,7 @@ def timed(fn, steps: int, stream, dist_on: bool, device):
     torch.cuda.synchronize(device)
     if dist_on:
         dist.barrier()
-    ms = t0.elapsed_time(t1)
-    if dist_on:
-        t = torch.tensor([ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(t0.elapsed_time(t1), device)
     return ms, launches, host_ms
 
 
@@ -308,6 +320,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--host-pool-gb", type=float, default=8.0)
     ap.add_argument("--jobs", default="", help="comma-separated subset of the workload's jobs (profiling a small case)")
+    ap.add_argument("--max-blocks", type=int, default=0, help="keep only the first N blocks of every job")
+    ap.add_argument("--chunk-elems", type=int, default=0, help="PS_OPT_CHUNK_ELEMS (0 = automatic)")
+    ap.add_argument("--kernel", type=int, default=0, help="PS_OPT_KERNEL (0 = automatic, 1 = direct loads, 2 = bulk-copy ring)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -320,6 +335,10 @@ def main():
     if args.jobs:
         cfg.jobs = [cfg.jobs[int(x)] for x in args.jobs.split(",")]
         cfg.name += "[jobs %s]" % args.jobs
+    if args.max_blocks:
+        for job in cfg.jobs:
+            job.blocks = job.blocks[:args.max_blocks]
+        cfg.name += "[first %d blocks]" % args.max_blocks
     config = {"workload": "%s: %d packed jobs, %d params, %d blocks, W=%s, %s arrival in <=%d rounds/step" % (
         cfg.name, len(cfg.jobs), cfg.num_params, sum(len(j.blocks) for j in cfg.jobs),
         sorted({j.num_workers for j in cfg.jobs}), cfg.arrival, args.ticks),
@@ -359,6 +378,8 @@ def main():
 
     n_sched = max(1, min(args.warmup + args.steps, 8))
     wl = Workload(cfg, local_rank, args.ticks, n_sched)
+    wl.svc.set_option(wl.B.PS_OPT_CHUNK_ELEMS, args.chunk_elems)
+    wl.svc.set_option(wl.B.PS_OPT_KERNEL, args.kernel)
     stream = torch.cuda.Stream(device)
 
     for k in range(args.warmup):
@@ -371,7 +392,7 @@ def main():
     clocks = sampler.stop() if rank == 0 else {}
     info = wl.svc.launch_info()
     assert info["launches"] - l0 == launches
-    value = world * wl.params_per_step * args.steps / (ms * 1e-3)
+    value = whole_job_value(wl.params_per_step, world, args.steps, ms)
     achieved = wl.bytes_per_step * args.steps / (ms * 1e-3) / 1e9     # per GPU
     peak, peak_kind = measured_peak()
     per_launch_bytes = wl.bytes_per_step * args.steps / launches
@@ -386,7 +407,7 @@ def main():
         wl.step_host(0, stream)         # warm-up: allocates the staging buffers
         torch.cuda.synchronize(device)
         ems, _, _ = timed(wl.step_host, args.e2e_steps, stream, dist_on, device)
-        e2e = {"value": world * wl.params_per_step * args.e2e_steps / (ems * 1e-3), "unit": UNIT,
+        e2e = {"value": whole_job_value(wl.params_per_step, world, args.e2e_steps, ems), "unit": UNIT,
                "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "steps": args.e2e_steps,
                "ms_per_step": ems / args.e2e_steps,
                "host_pool_bytes": wl.pool_bytes}

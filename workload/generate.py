@@ -58,6 +58,8 @@ def _apply_row_sparsity(spec: JobSpec, row: torch.Tensor, gen: torch.Generator):
     off = 0
     for t in spec.tensors:
         n = t.nelem
+        if off + n > row.numel():     # job truncated to its first blocks (profiling)
+            break
         if t.row_sparse:
             rows = t.shape[0]
             keep = torch.rand(rows, generator=gen, device=row.device) < spec.sparse_row_fraction
