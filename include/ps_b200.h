@@ -75,12 +75,12 @@ typedef struct { int job, block; } ps_task;
 
 /* Options for ps_set_option / ps_get_option. */
 enum {
-  PS_OPT_CHUNK_ELEMS = 1,  /* elements per (job,block,chunk) descriptor; 0 = automatic.
+  PS_OPT_CHUNK_ELEMS = 1,  /* elements per (job,block,chunk) descriptor; 0 = automatic (8192).
                               Must be a multiple of 1024 (<= 2^20) when non-zero. */
   PS_OPT_CTAS_PER_SM = 2,  /* persistent CTAs per SM; 0 = automatic */
   PS_OPT_SORT_TASKS = 3,   /* 1 (default): heaviest chunks first inside a launch; 0: caller's order */
-  PS_OPT_KERNEL = 4        /* kernel variant: 0 = automatic (currently direct loads), 1 = direct
-                              loads, 2 = bulk-copy ring; results are identical except for the
+  PS_OPT_KERNEL = 4        /* kernel variant: 0 = automatic (direct loads), 1 = direct loads,
+                              2 = bulk-copy ring; results are identical except for the
                               rounding of the per-block norm */
 };
 

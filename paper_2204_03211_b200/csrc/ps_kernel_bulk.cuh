@@ -144,7 +144,7 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
   PsTaskDev* tasks = reinterpret_cast<PsTaskDev*>(table + hdr->tasks_off);
   const unsigned int* starts = reinterpret_cast<const unsigned int*>(table + hdr->starts_off);
   const void* const* ptrs = reinterpret_cast<const void* const*>(table + hdr->ptrs_off);
-  const unsigned int n_tasks = hdr->n_tasks, total = hdr->total_chunks, chunk_elems = hdr->chunk_elems;
+  const unsigned int n_tasks = hdr->n_tasks, total = hdr->total_chunks;
 
   const unsigned int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
@@ -175,6 +175,7 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
       const unsigned int ges = J->grad_dtype ? 2u : 4u;
       const unsigned int vecw = J->grad_dtype ? 8u : 4u;
       const int nstate = J->opt ? 2 : 1;
+      const unsigned int chunk_elems = T->chunk_elems;
       const size_t begin = (size_t)(idx - T->first_chunk) * chunk_elems;
       const unsigned int count = (unsigned int)min((unsigned long long)chunk_elems, T->nelem - begin);
       const unsigned int tile = T->tile_elems;
@@ -277,6 +278,7 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
       kind = (J->opt << 1) | J->grad_dtype;
       p = T->p; s0 = T->s0; s1 = T->s1;
     }
+    const unsigned int chunk_elems = T->chunk_elems;
     const size_t begin = (size_t)(m.chunk - T->first_chunk) * chunk_elems;
     const unsigned int count = (unsigned int)min((unsigned long long)chunk_elems, T->nelem - begin);
     if (m.flags & kTileDirect) {

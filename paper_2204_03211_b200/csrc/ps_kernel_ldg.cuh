@@ -17,7 +17,7 @@ ps_aggregate_ldg_kernel(unsigned char* __restrict__ table, const PsJobDev* __res
   PsTaskDev* tasks = reinterpret_cast<PsTaskDev*>(table + hdr->tasks_off);
   const unsigned int* starts = reinterpret_cast<const unsigned int*>(table + hdr->starts_off);
   const void* const* ptrs = reinterpret_cast<const void* const*>(table + hdr->ptrs_off);
-  const unsigned int n_tasks = hdr->n_tasks, total = hdr->total_chunks, chunk_elems = hdr->chunk_elems;
+  const unsigned int n_tasks = hdr->n_tasks, total = hdr->total_chunks;
 
   __shared__ unsigned int s_idx[2];
   __shared__ unsigned int s_task;
@@ -42,6 +42,7 @@ ps_aggregate_ldg_kernel(unsigned char* __restrict__ table, const PsJobDev* __res
 
     const unsigned int t = s_task;
     const PsTaskDev* T = tasks + t;
+    const unsigned int chunk_elems = T->chunk_elems;
     const size_t begin = (size_t)(idx - T->first_chunk) * chunk_elems;
     const unsigned int count = (unsigned int)min((unsigned long long)chunk_elems, T->nelem - begin);
     double sq = 0.0;

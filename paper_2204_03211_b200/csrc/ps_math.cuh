@@ -34,9 +34,10 @@ __device__ __forceinline__ void update_elem(const Hp& h, float G, float& p, floa
 __device__ __forceinline__ float bf16_lo(unsigned int u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(unsigned int u) { return __uint_as_float(u & 0xffff0000u); }
 
-// Shard pointer w of a task, through the read-only path (uniform across the CTA).
+// Shard pointer w of a task (uniform across the CTA).  A generic load: the
+// pointer row may sit in the global task table or in shared memory.
 __device__ __forceinline__ const void* ld_ptr(const void* const* shards, int w = 0) {
-  return reinterpret_cast<const void*>(__ldg(reinterpret_cast<const unsigned long long*>(shards) + w));
+  return shards[w];
 }
 
 // Streaming (read-once) 128-bit load.

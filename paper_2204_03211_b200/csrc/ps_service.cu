@@ -75,6 +75,7 @@ struct Slot {
   double* partials = nullptr;
   size_t partial_cap = 0;
   cudaEvent_t done = nullptr;
+  cudaEvent_t copied = nullptr;            // table upload finished (recorded on the copy stream)
   bool inflight = false;
   unsigned long long gen = 0;
 };
@@ -107,6 +108,7 @@ struct ps_service {
   unsigned long long gen = 0;              // ready-list generation
   long long opt_chunk = 0, opt_ctas = 0, opt_sort = 1, opt_kernel = 0;
   int* status_dev = nullptr;               // error word written by kernels whose waits expired
+  cudaStream_t copy_stream = nullptr;      // table uploads run here, beside the previous launch
   int occ_ctas = 0;
   unsigned long long launches = 0;
   int last_grid = 0, last_block = 0;
@@ -219,28 +221,25 @@ int validate_ready(ps_service* s, const ps_task* ready, int n_ready, std::vector
 
 size_t bytes_per_elem(const Job& j) { return (size_t)j.d.num_workers * j.grad_esize() + 8 * (1 + j.nstate()); }
 
-// Automatic = the direct-load kernel: measured faster than the bulk-copy ring
-// on every configuration so far.
-bool use_bulk(const ps_service* s) { return s->opt_kernel == 2; }
+// Kernel variants (PS_OPT_KERNEL): 1 direct loads, 2 bulk-copy ring.
+// Automatic = 1, measured faster on every configuration so far.
+enum { kKernelLdg = 1, kKernelBulk = 2 };
+int kernel_of(const ps_service* s) { return s->opt_kernel == 0 ? kKernelLdg : (int)s->opt_kernel; }
+bool use_bulk(const ps_service* s) { return kernel_of(s) == kKernelBulk; }
 
 int grid_cap(ps_service* s) {
   int per_sm;
   if (use_bulk(s)) per_sm = 1;   // one warp-specialised CTA owns an SM's shared memory
-  else per_sm = s->opt_ctas > 0 ? (int)s->opt_ctas : (s->occ_ctas > 0 ? s->occ_ctas : 3);
+  else if (s->opt_ctas > 0) per_sm = (int)s->opt_ctas;
+  else per_sm = s->occ_ctas > 0 ? s->occ_ctas : 3;
   return s->num_sms * per_sm;
 }
 
-unsigned int pick_chunk_elems(ps_service* s, const std::vector<int>& idx) {
-  if (s->opt_chunk > 0) return (unsigned int)s->opt_chunk;
-  // Aim for ~16 chunks per resident CTA so that the tail of a launch is short,
-  // within [2048, 8192] elements.
-  unsigned long long total = 0;
-  for (int bi : idx) total += s->blocks[bi].nelem;
-  unsigned long long want = total / ((unsigned long long)grid_cap(s) * 16ull);
-  unsigned int c = 8192;
-  while (c > 2048 && c > want) c >>= 1;
-  return c;
-}
+// Automatic chunk size.  Measured on B200 (C2, C4 all-ready and C4 in bursty
+// rounds): 8192 elements beats 2048/4096/16384 and beats shrinking the chunks
+// toward the end of the table; the per-launch cost that remains (about 30 us)
+// is launch latency, ramp-up and the last wave, not chunk bookkeeping.
+constexpr unsigned int kChunkAuto = 8192;
 
 // Elements per ring tile of the bulk-copy kernel: the largest multiple of 128
 // whose rows (W shards, parameters, state) fit one stage; 0 if none does.
@@ -254,8 +253,9 @@ unsigned int tile_elems_for(const Job& j) {
 int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
   const size_t n = idx.size();
   plan->order = idx;
-  plan->chunk_elems = pick_chunk_elems(s, idx);
-  const unsigned int ce = plan->chunk_elems;
+  const bool fixed = s->opt_chunk > 0;
+  const unsigned int ce = fixed ? (unsigned int)s->opt_chunk : kChunkAuto;
+  plan->chunk_elems = ce;
   if (s->opt_sort) {
     // heaviest chunks first: the launch's tail is then made of light chunks
     std::stable_sort(plan->order.begin(), plan->order.end(), [&](int a, int b) {
@@ -268,6 +268,7 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
   }
   size_t nptr = 0;
   for (int bi : plan->order) nptr += s->jobs[s->blocks[bi].job].d.num_workers;
+
   const size_t tasks_off = sizeof(PsTableHdr);
   const size_t starts_off = tasks_off + n * sizeof(PsTaskDev);
   const size_t ptrs_off = (starts_off + n * sizeof(unsigned int) + 15) / 16 * 16;
@@ -288,7 +289,8 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
     t.nelem = b.nelem;
     t.shard_row = (unsigned int)row;
     t.first_chunk = (unsigned int)chunk;
-    t.nchunks = (unsigned int)((b.nelem + ce - 1) / ce);
+    t.chunk_elems = ce;
+    t.nchunks = (unsigned int)((b.nelem + t.chunk_elems - 1) / t.chunk_elems);
     t.ticket = 0;
     const unsigned long long step = b.step + 1;
     t.ss_t = (float)((double)j.d.lr / (1.0 - std::pow((double)j.d.beta1, (double)step)));
@@ -328,6 +330,7 @@ int acquire_slot(ps_service* s, size_t table_bytes, size_t nchunks, Slot** out) 
     sl.inflight = false;
   }
   if (!sl.done) PS_CUDA(s, cudaEventCreateWithFlags(&sl.done, cudaEventDisableTiming));
+  if (!sl.copied) PS_CUDA(s, cudaEventCreateWithFlags(&sl.copied, cudaEventDisableTiming));
   if (table_bytes > sl.cap) {
     size_t ncap = std::max<size_t>(table_bytes * 2, 1 << 16);
     if (sl.host) PS_CUDA(s, cudaFreeHost(sl.host));
@@ -395,6 +398,7 @@ int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes
       e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&s->occ_ctas, ps_aggregate_ldg_kernel, kThreads, 0);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(ps_aggregate_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBulkSmemBytes);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaMalloc(&s->status_dev, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(s->status_dev, 0, sizeof(int));
     for (int c = 0; e == cudaSuccess && c < num_contexts; ++c) {
@@ -406,6 +410,7 @@ int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes
       const bool oom = (e == cudaErrorMemoryAllocation);
       for (auto& c : s->ctxs) if (c.base) cudaFree(c.base);
       if (s->status_dev) cudaFree(s->status_dev);
+      if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
       cudaGetLastError();
       delete s;
       return oom ? PS_ERR_NOMEM : PS_ERR_CUDA;
@@ -429,11 +434,13 @@ int ps_destroy(ps_service* s) {
       if (sl.dev) cudaFree(sl.dev);
       if (sl.partials) cudaFree(sl.partials);
       if (sl.done) cudaEventDestroy(sl.done);
+      if (sl.copied) cudaEventDestroy(sl.copied);
     }
     for (auto& c : s->ctxs) if (c.base) cudaFree(c.base);
     if (s->jobs_dev) cudaFree(s->jobs_dev);
     if (s->stats_dev) cudaFree(s->stats_dev);
     if (s->status_dev) cudaFree(s->status_dev);
+    if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
   }
   s->magic = 0;
   delete s;
@@ -586,7 +593,11 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
     if (rc) return rc;
   }
   std::memcpy(sl->host, plan.bytes.data(), plan.bytes.size());
-  PS_CUDA(s, cudaMemcpyAsync(sl->dev, sl->host, plan.bytes.size(), cudaMemcpyHostToDevice, stream));
+  // The table depends on nothing the caller enqueued, so its upload goes to the
+  // service's own stream and overlaps the previous launch; the kernel waits for it.
+  PS_CUDA(s, cudaMemcpyAsync(sl->dev, sl->host, plan.bytes.size(), cudaMemcpyHostToDevice, s->copy_stream));
+  PS_CUDA(s, cudaEventRecord(sl->copied, s->copy_stream));
+  PS_CUDA(s, cudaStreamWaitEvent(stream, sl->copied, 0));
   const int grid = (int)std::min<unsigned long long>(plan.total_chunks, (unsigned long long)grid_cap(s));
   if (bulk)
     ps_aggregate_bulk_kernel<<<grid, kBulkThreads, kBulkSmemBytes, stream>>>(sl->dev, s->jobs_dev, s->stats_dev,
@@ -636,8 +647,8 @@ int ps_plan(ps_service* s, const ps_task* ready, int n_ready, ps_chunk_info* out
       ps_chunk_info& ci = out[k];
       ci.job = b.job;
       ci.block = b.id;
-      ci.elem_begin = (unsigned long long)c * h->chunk_elems;
-      ci.elem_count = std::min<unsigned long long>(h->chunk_elems, tasks[t].nelem - ci.elem_begin);
+      ci.elem_begin = (unsigned long long)c * tasks[t].chunk_elems;
+      ci.elem_count = std::min<unsigned long long>(tasks[t].chunk_elems, tasks[t].nelem - ci.elem_begin);
       ci.num_workers = s->jobs[b.job].d.num_workers;
       ci.vector_path = (int)tasks[t].vec_ok;
     }
@@ -867,10 +878,10 @@ namespace psb {
 constexpr unsigned int kNaChunk = 8192;                                   // elements per chunk
 constexpr size_t kNaMaxChunks = PS_NOALLOC_MAX_ELEMS / kNaChunk;          // 2048
 constexpr size_t kNaTaskOff = sizeof(PsTableHdr);                         // 32
-constexpr size_t kNaStartsOff = kNaTaskOff + sizeof(PsTaskDev);           // 112
-constexpr size_t kNaPtrsOff = 128;
-constexpr size_t kNaJobOff = kNaPtrsOff + PS_MAX_WORKERS * sizeof(void*); // 2176
-constexpr size_t kNaStatOff = kNaJobOff + sizeof(PsJobDev);               // 2240
+constexpr size_t kNaStartsOff = kNaTaskOff + sizeof(PsTaskDev);           // 128
+constexpr size_t kNaPtrsOff = 144;
+constexpr size_t kNaJobOff = kNaPtrsOff + PS_MAX_WORKERS * sizeof(void*); // 2192
+constexpr size_t kNaStatOff = kNaJobOff + sizeof(PsJobDev);               // 2256
 constexpr size_t kNaPartOff = 2304;
 constexpr size_t kNaScratchBytes = kNaPartOff + kNaMaxChunks * sizeof(double);   // 18688
 static_assert(kNaStartsOff + sizeof(unsigned int) <= kNaPtrsOff, "scratch layout");
@@ -986,6 +997,7 @@ extern "C" int ps_aggregate_block_noalloc(const ps_job_desc* job, unsigned long 
   a.task.step = step;
   a.task.vec_ok = (all & 15u) ? 0u : 1u;
   a.task.tile_elems = 0;
+  a.task.chunk_elems = kNaChunk;
   for (int w = 0; w < job->num_workers; ++w) a.shards[w] = shard_ptrs[w];
 
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);

@@ -21,7 +21,7 @@ struct __align__(16) PsJobDev {        // 64 bytes, one per registered job
   float lr, mom, wd, b1, b2, omb1, omb2, eps, gs, _r0, _r1, _r2;
 };
 
-struct __align__(16) PsTaskDev {       // 80 bytes, one per ready (job, block)
+struct __align__(16) PsTaskDev {       // 96 bytes, one per ready (job, block)
   float* p;
   float* s0;
   float* s1;
@@ -36,13 +36,15 @@ struct __align__(16) PsTaskDev {       // 80 bytes, one per ready (job, block)
   unsigned long long step;
   unsigned int vec_ok;                 // all pointers 16-byte aligned
   unsigned int tile_elems;             // elements per ring tile (bulk-copy kernel); 0 = direct loads only
+  unsigned int chunk_elems;            // elements per chunk of THIS task (multiple of 1024)
+  unsigned int _r0, _r1, _r2;
 };
 
 struct __align__(16) PsTableHdr {      // 32 bytes at the start of the table
   unsigned int counter;                // next chunk to claim (uploaded as 0)
   unsigned int n_tasks;
   unsigned int total_chunks;
-  unsigned int chunk_elems;
+  unsigned int chunk_elems;            // largest chunk size used in this table
   unsigned int tasks_off, starts_off, ptrs_off;   // byte offsets from the table base
   unsigned int parts_per_chunk;        // partial sums each chunk publishes (1 per CTA or 1 per consumer warp)
 };
