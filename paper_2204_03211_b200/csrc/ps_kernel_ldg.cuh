@@ -10,7 +10,7 @@ namespace psb {
 
 constexpr int kThreads = 256;          // threads per CTA
 
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, 4)
 ps_aggregate_ldg_kernel(unsigned char* __restrict__ table, const PsJobDev* __restrict__ jobs,
                         PsStat* __restrict__ stats, double* __restrict__ partials) {
   PsTableHdr* hdr = reinterpret_cast<PsTableHdr*>(table);
