@@ -79,6 +79,8 @@ enum {
                               Must be a multiple of 1024 (<= 2^20) when non-zero. */
   PS_OPT_CTAS_PER_SM = 2,  /* persistent CTAs per SM; 0 = automatic */
   PS_OPT_SORT_TASKS = 3,   /* 1 (default): heaviest chunks first inside a launch; 0: caller's order */
+  PS_OPT_PROFILE = 5,      /* 1: aggregates record per-task device time (see ps_block_profile);
+                              costs a few atomics per chunk; direct-load kernel only; default 0 */
   PS_OPT_KERNEL = 4        /* kernel variant: 0 = automatic (direct loads), 1 = direct loads,
                               2 = bulk-copy ring; results are identical except for the
                               rounding of the per-block norm */
@@ -178,6 +180,21 @@ int ps_migrate_block(ps_service* svc, int job, int block, int dst_ctx, void* str
  * NULL.  Before the first aggregate the norm is 0 and the step 0. */
 int ps_block_stats(ps_service* svc, int job, int block, double* grad_sqnorm_out,
                    unsigned long long* step_out);
+
+/* Device time of the block's last aggregate, recorded when PS_OPT_PROFILE was on
+ * for that launch (zeros otherwise) — the counterpart of the per-task execution
+ * time e_t that the paper's profilers collect for the assignment scheme
+ * (Section 3.1; Pseudocode 1 takes e_t as input).  busy = sum over the task's
+ * chunks of the time a CTA spent on the chunk (CTA-microseconds; chunks of one
+ * task run concurrently on many CTAs); span = last chunk end - first chunk
+ * start.  Timer: the GPU's %globaltimer (resolution is device dependent, up to
+ * about 1 us).  Waits for the block's last aggregate.  Out pointers may be NULL. */
+int ps_block_profile(ps_service* svc, int job, int block, double* busy_us_out, double* span_us_out);
+
+/* The same over all blocks of a job (each block's last aggregate): summed busy
+ * time, span from the earliest chunk start to the latest chunk end, and the
+ * number of blocks that carried a profile. */
+int ps_job_profile(ps_service* svc, int job, double* busy_us_out, double* span_us_out, int* blocks_out);
 
 /* Device pointers to the block's optimizer state (momentum | Adam m, and
  * Adam v or NULL) and its current context; for tests and checkpoints. */

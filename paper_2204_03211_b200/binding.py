@@ -23,7 +23,7 @@ PS_ERR_TOO_LARGE = -9
 PS_NOALLOC_MAX_ELEMS = 1 << 24
 PS_DEVICE_NONE = -1
 PS_MAX_WORKERS = 256
-PS_OPT_CHUNK_ELEMS, PS_OPT_CTAS_PER_SM, PS_OPT_SORT_TASKS, PS_OPT_KERNEL = 1, 2, 3, 4
+PS_OPT_CHUNK_ELEMS, PS_OPT_CTAS_PER_SM, PS_OPT_SORT_TASKS, PS_OPT_KERNEL, PS_OPT_PROFILE = 1, 2, 3, 4, 5
 
 
 class ps_job_desc(C.Structure):
@@ -64,6 +64,9 @@ _SIGNATURES = {
     "ps_pull_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
     "ps_migrate_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]),
     "ps_block_stats": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_ulonglong)]),
+    "ps_block_profile": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double)]),
+    "ps_job_profile": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                 C.POINTER(C.c_int)]),
     "ps_block_state": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p),
                                  C.POINTER(C.c_int)]),
     "ps_plan": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]),
@@ -209,6 +212,18 @@ def ps_block_stats(svc, job: int, block: int):
     return sq.value, step.value
 
 
+def ps_block_profile(svc, job: int, block: int):
+    busy, span = C.c_double(), C.c_double()
+    _check(load().ps_block_profile(svc, job, block, C.byref(busy), C.byref(span)), "ps_block_profile", svc)
+    return busy.value, span.value
+
+
+def ps_job_profile(svc, job: int):
+    busy, span, n = C.c_double(), C.c_double(), C.c_int()
+    _check(load().ps_job_profile(svc, job, C.byref(busy), C.byref(span), C.byref(n)), "ps_job_profile", svc)
+    return busy.value, span.value, n.value
+
+
 def ps_block_state(svc, job: int, block: int):
     s0, s1, ctx = C.c_void_p(), C.c_void_p(), C.c_int()
     _check(load().ps_block_state(svc, job, block, C.byref(s0), C.byref(s1), C.byref(ctx)), "ps_block_state", svc)
@@ -314,6 +329,6 @@ def _bind(name):
 
 
 for _n in ("register_job", "register_block", "push", "push_batch", "push_host", "aggregate", "pull", "pull_batch", "pull_host",
-           "migrate_block", "block_stats", "block_state", "plan", "set_option", "get_option", "arena_info",
+           "migrate_block", "block_stats", "block_profile", "job_profile", "block_state", "plan", "set_option", "get_option", "arena_info",
            "launch_info", "device_status"):
     setattr(Service, _n, _bind(_n))

@@ -18,6 +18,7 @@ ps_aggregate_ldg_kernel(unsigned char* __restrict__ table, const PsJobDev* __res
   const unsigned int* starts = reinterpret_cast<const unsigned int*>(table + hdr->starts_off);
   const void* const* ptrs = reinterpret_cast<const void* const*>(table + hdr->ptrs_off);
   const unsigned int n_tasks = hdr->n_tasks, total = hdr->total_chunks;
+  const bool profile = hdr->profile != 0;
 
   __shared__ unsigned int s_idx[2];
   __shared__ unsigned int s_task;
@@ -40,6 +41,7 @@ ps_aggregate_ldg_kernel(unsigned char* __restrict__ table, const PsJobDev* __res
     }
     __syncthreads();
 
+    const unsigned long long t_begin = (profile && tid == 0) ? global_ns() : 0ull;
     const unsigned int t = s_task;
     const PsTaskDev* T = tasks + t;
     const unsigned int chunk_elems = T->chunk_elems;
@@ -57,6 +59,7 @@ ps_aggregate_ldg_kernel(unsigned char* __restrict__ table, const PsJobDev* __res
       double s = s_red[0];
 #pragma unroll
       for (int k = 1; k < kThreads / 32; ++k) s += s_red[k];
+      if (profile) profile_chunk(tasks + t, t_begin, global_ns());
       publish_part(tasks, t, idx, 1u, s, stats, partials);
     }
     buf ^= 1;

@@ -233,8 +233,27 @@ __device__ __forceinline__ void publish_part(PsTaskDev* tasks, unsigned int t, u
     PsStat st;
     st.sqnorm = tot;
     st.step = T->step;
+    st.busy_ns = __ldcg(&T->busy_ns);
+    const unsigned long long tf = __ldcg(&T->t_first);
+    st.t_first = (tf == ~0ull) ? 0ull : tf;
+    st.t_last = __ldcg(&T->t_last);
+    st._r0 = 0;
     stats[T->stat_idx] = st;
   }
+}
+
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Adds one chunk's device time to its task's profile (before publish_part, whose
+// fence orders these updates ahead of the ticket).
+__device__ __forceinline__ void profile_chunk(PsTaskDev* T, unsigned long long t0, unsigned long long t1) {
+  atomicAdd(&T->busy_ns, t1 - t0);
+  atomicMin(&T->t_first, t0);
+  atomicMax(&T->t_last, t1);
 }
 
 // Advances `cursor` (uniform in the calling warp) to the task that owns chunk

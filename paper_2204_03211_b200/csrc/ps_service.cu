@@ -106,7 +106,7 @@ struct ps_service {
   Slot slots[kSlots];
   int next_slot = 0;
   unsigned long long gen = 0;              // ready-list generation
-  long long opt_chunk = 0, opt_ctas = 0, opt_sort = 1, opt_kernel = 0;
+  long long opt_chunk = 0, opt_ctas = 0, opt_sort = 1, opt_kernel = 0, opt_profile = 0;
   int* status_dev = nullptr;               // error word written by kernels whose waits expired
   cudaStream_t copy_stream = nullptr;      // table uploads run here, beside the previous launch
   int occ_ctas = 0;
@@ -292,6 +292,9 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
     t.chunk_elems = ce;
     t.nchunks = (unsigned int)((b.nelem + t.chunk_elems - 1) / t.chunk_elems);
     t.ticket = 0;
+    t.busy_ns = 0;
+    t.t_first = ~0ull;
+    t.t_last = 0;
     const unsigned long long step = b.step + 1;
     t.ss_t = (float)((double)j.d.lr / (1.0 - std::pow((double)j.d.beta1, (double)step)));
     t.sbc2_t = (float)std::sqrt(1.0 - std::pow((double)j.d.beta2, (double)step));
@@ -320,6 +323,7 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
   h->starts_off = (unsigned int)starts_off;
   h->ptrs_off = (unsigned int)ptrs_off;
   h->parts_per_chunk = use_bulk(s) ? kBulkConsumerWarps : 1;
+  h->profile = s->opt_profile ? 1u : 0u;
   return PS_OK;
 }
 
@@ -755,6 +759,54 @@ int ps_block_stats(ps_service* s, int job, int block, double* sq_out, unsigned l
   return PS_OK;
 }
 
+// Waits for the block's last aggregate and reads its statistics record.
+static int read_stat(ps_service* s, Block& b, PsStat* st) {
+  std::memset(st, 0, sizeof *st);
+  if (!has_device(s) || b.last_slot < 0) return PS_OK;
+  PS_CUDA(s, cudaSetDevice(s->device));
+  Slot& sl = s->slots[b.last_slot];
+  if (sl.inflight && sl.gen == b.last_slot_gen) PS_CUDA(s, cudaEventSynchronize(sl.done));
+  PS_CUDA(s, cudaMemcpy(st, s->stats_dev + b.stat_idx, sizeof *st, cudaMemcpyDeviceToHost));
+  return PS_OK;
+}
+
+int ps_block_profile(ps_service* s, int job, int block, double* busy_us_out, double* span_us_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  const int bi = find_block(s, job, block);
+  if (bi < 0) return PS_ERR_BAD_ARG;
+  PsStat st;
+  int rc = read_stat(s, s->blocks[bi], &st);
+  if (rc) return rc;
+  if (busy_us_out) *busy_us_out = st.busy_ns * 1e-3;
+  if (span_us_out) *span_us_out = st.t_last > st.t_first ? (st.t_last - st.t_first) * 1e-3 : 0.0;
+  return PS_OK;
+}
+
+int ps_job_profile(ps_service* s, int job, double* busy_us_out, double* span_us_out, int* blocks_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (job < 0 || job >= (int)s->jobs.size()) return PS_ERR_BAD_ARG;
+  double busy = 0.0;
+  unsigned long long first = ~0ull, last = 0;
+  int n = 0;
+  for (int bi : s->jobs[job].block_of_id) {
+    if (bi < 0) continue;
+    PsStat st;
+    int rc = read_stat(s, s->blocks[bi], &st);
+    if (rc) return rc;
+    if (st.t_last == 0) continue;          // never profiled
+    busy += st.busy_ns * 1e-3;
+    first = std::min(first, st.t_first);
+    last = std::max(last, st.t_last);
+    ++n;
+  }
+  if (busy_us_out) *busy_us_out = busy;
+  if (span_us_out) *span_us_out = n && last > first ? (last - first) * 1e-3 : 0.0;
+  if (blocks_out) *blocks_out = n;
+  return PS_OK;
+}
+
 int ps_block_state(ps_service* s, int job, int block, const float** s0, const float** s1, int* ctx_out) {
   if (!alive(s)) return PS_ERR_BAD_HANDLE;
   std::lock_guard<std::mutex> lk(s->mu);
@@ -786,6 +838,9 @@ int ps_set_option(ps_service* s, int option, long long value) {
       if (value < 0 || value > 2) return PS_ERR_BAD_ARG;
       s->opt_kernel = value;
       return PS_OK;
+    case PS_OPT_PROFILE:
+      s->opt_profile = value ? 1 : 0;
+      return PS_OK;
     default:
       return PS_ERR_BAD_ARG;
   }
@@ -800,6 +855,7 @@ int ps_get_option(ps_service* s, int option, long long* out) {
     case PS_OPT_CTAS_PER_SM: *out = s->opt_ctas; return PS_OK;
     case PS_OPT_SORT_TASKS: *out = s->opt_sort; return PS_OK;
     case PS_OPT_KERNEL: *out = s->opt_kernel; return PS_OK;
+    case PS_OPT_PROFILE: *out = s->opt_profile; return PS_OK;
     default: return PS_ERR_BAD_ARG;
   }
 }
@@ -877,12 +933,12 @@ namespace psb {
 
 constexpr unsigned int kNaChunk = 8192;                                   // elements per chunk
 constexpr size_t kNaMaxChunks = PS_NOALLOC_MAX_ELEMS / kNaChunk;          // 2048
-constexpr size_t kNaTaskOff = sizeof(PsTableHdr);                         // 32
-constexpr size_t kNaStartsOff = kNaTaskOff + sizeof(PsTaskDev);           // 128
-constexpr size_t kNaPtrsOff = 144;
-constexpr size_t kNaJobOff = kNaPtrsOff + PS_MAX_WORKERS * sizeof(void*); // 2192
-constexpr size_t kNaStatOff = kNaJobOff + sizeof(PsJobDev);               // 2256
-constexpr size_t kNaPartOff = 2304;
+constexpr size_t kNaTaskOff = sizeof(PsTableHdr);                         // 48
+constexpr size_t kNaStartsOff = kNaTaskOff + sizeof(PsTaskDev);           // 176
+constexpr size_t kNaPtrsOff = 192;
+constexpr size_t kNaJobOff = kNaPtrsOff + PS_MAX_WORKERS * sizeof(void*); // 2240
+constexpr size_t kNaStatOff = kNaJobOff + sizeof(PsJobDev);               // 2304
+constexpr size_t kNaPartOff = 2560;
 constexpr size_t kNaScratchBytes = kNaPartOff + kNaMaxChunks * sizeof(double);   // 18688
 static_assert(kNaStartsOff + sizeof(unsigned int) <= kNaPtrsOff, "scratch layout");
 static_assert(kNaStatOff + sizeof(PsStat) <= kNaPartOff, "scratch layout");
@@ -913,6 +969,8 @@ __global__ void ps_noalloc_setup_kernel(NoAllocArgs a) {
     h.starts_off = (unsigned int)kNaStartsOff;
     h.ptrs_off = (unsigned int)kNaPtrsOff;
     h.parts_per_chunk = 1;
+    h.profile = 0;
+    h._r0 = h._r1 = h._r2 = 0;
     *reinterpret_cast<PsTableHdr*>(base) = h;
     *reinterpret_cast<PsTaskDev*>(base + kNaTaskOff) = a.task;     // ticket = 0 inside
     *reinterpret_cast<unsigned int*>(base + kNaStartsOff) = 0;
@@ -920,6 +978,7 @@ __global__ void ps_noalloc_setup_kernel(NoAllocArgs a) {
     PsStat z;
     z.sqnorm = 0.0;
     z.step = 0;
+    z.busy_ns = z.t_first = z.t_last = z._r0 = 0;
     *reinterpret_cast<PsStat*>(base + kNaStatOff) = z;
   }
 }

@@ -21,7 +21,7 @@ struct __align__(16) PsJobDev {        // 64 bytes, one per registered job
   float lr, mom, wd, b1, b2, omb1, omb2, eps, gs, _r0, _r1, _r2;
 };
 
-struct __align__(16) PsTaskDev {       // 96 bytes, one per ready (job, block)
+struct __align__(16) PsTaskDev {       // 128 bytes, one per ready (job, block)
   float* p;
   float* s0;
   float* s1;
@@ -38,20 +38,29 @@ struct __align__(16) PsTaskDev {       // 96 bytes, one per ready (job, block)
   unsigned int tile_elems;             // elements per ring tile (bulk-copy kernel); 0 = direct loads only
   unsigned int chunk_elems;            // elements per chunk of THIS task (multiple of 1024)
   unsigned int _r0, _r1, _r2;
+  // device-time profile of this task, filled only when the table asks for it
+  unsigned long long busy_ns;          // sum over chunks of (chunk end - chunk start)      (uploaded as 0)
+  unsigned long long t_first;          // earliest chunk start, %globaltimer ns             (uploaded as ~0)
+  unsigned long long t_last;           // latest chunk end                                  (uploaded as 0)
+  unsigned long long _r3;
 };
 
-struct __align__(16) PsTableHdr {      // 32 bytes at the start of the table
+struct __align__(16) PsTableHdr {      // 48 bytes at the start of the table
   unsigned int counter;                // next chunk to claim (uploaded as 0)
   unsigned int n_tasks;
   unsigned int total_chunks;
   unsigned int chunk_elems;            // largest chunk size used in this table
   unsigned int tasks_off, starts_off, ptrs_off;   // byte offsets from the table base
   unsigned int parts_per_chunk;        // partial sums each chunk publishes (1 per CTA or 1 per consumer warp)
+  unsigned int profile;                // 1: record per-task device time (direct-load kernel)
+  unsigned int _r0, _r1, _r2;
 };
 
-struct __align__(16) PsStat {
+struct __align__(16) PsStat {          // 48 bytes per registered block, written by the task's last chunk
   double sqnorm;
   unsigned long long step;
+  unsigned long long busy_ns, t_first, t_last;   // zero unless profiling was on
+  unsigned long long _r0;
 };
 
 }  // namespace psb
