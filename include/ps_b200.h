@@ -268,6 +268,53 @@ int ps_aggregate_block_noalloc(const ps_job_desc* job, unsigned long long step, 
                                const void* const* shard_dev_ptrs, double* sqnorm_dev_out_or_null,
                                void* stream);
 
+/* ---------------------------------------------------------------------------
+ * Planner: which Aggregator (context) runs which aggregation task.  Host only.
+ *
+ * The paper's assignment heuristic — Section 3.3.1, Pseudocode 1 "Model
+ * Aggregation Assignment Scheme" — with cyclic execution: an Aggregator's cycle
+ * C_n is the largest iteration duration D_j among its jobs; job j gets a slot
+ * every d_j = max(D_j, C_n / floor(C_n / D_j)); a destination is dropped when a
+ * job on it (or the new task's job) would lose (d_j - D_j)/d_j >= loss_limit;
+ * among the rest the task goes to the best fit, i.e. the Aggregator with the
+ * fewest free slots F_n = C_n - sum_j floor(C_n/d_j) * sum_{t of j on n} e_t that
+ * still hold the task's floor(C_n/d_k) * e_t; if none, a new Aggregator is
+ * allocated.  Times are in any one unit (e.g. microseconds from
+ * ps_block_profile for e_t, the job's measured iteration period for D_j).
+ * Aggregator indices count from 0 and are meant to be used as `ctx` in
+ * ps_register_block / ps_migrate_block.
+ * ------------------------------------------------------------------------- */
+typedef struct ps_planner ps_planner; /* opaque */
+
+/* loss_limit: the paper's LossLimit (default 0.1), in (0, 1]. */
+int ps_planner_create(ps_planner** out, double loss_limit);
+int ps_planner_destroy(ps_planner* pl);
+/* Registers a job with profiled iteration duration D_j > 0. */
+int ps_planner_add_job(ps_planner* pl, double iter_duration, int* job_out);
+/* Pseudocode 1 for one new task of `job` with execution time e_t > 0: chooses
+ * (or allocates) an Aggregator and records the assignment. */
+int ps_planner_assign(ps_planner* pl, int job, double exec_time, int* task_out, int* aggregator_out);
+/* Job exit (Section 3.3.2): drops the job's tasks, releases Aggregators left
+ * empty, then repeatedly tries to empty the least-loaded Aggregator by
+ * re-assigning its tasks to the others without new allocations; stops at the
+ * first one that cannot be emptied (its tasks stay).  Released Aggregators keep
+ * their index and are never reused.  Tasks that moved report their new
+ * Aggregator through ps_planner_task_info (the caller migrates the blocks). */
+int ps_planner_remove_job(ps_planner* pl, int job, int* released_out);
+int ps_planner_task_info(ps_planner* pl, int task, int* job_out, int* aggregator_out, double* exec_time_out);
+/* cycle = C_n; load = W_n = sum_j floor(C_n/d_j) * sum e_t (Appendix C). */
+int ps_planner_aggregator_info(ps_planner* pl, int aggregator, int* alive_out, double* cycle_out,
+                               double* load_out, int* num_tasks_out);
+/* D_j, the current d_j (largest over the Aggregators that hold its tasks) and
+ * the loss (d_j - D_j)/d_j. */
+int ps_planner_job_info(ps_planner* pl, int job, double* profiled_out, double* current_out, double* loss_out);
+int ps_planner_num_aggregators(ps_planner* pl, int* allocated_out, int* alive_out);
+/* Late request ("Handling Outliers in Cyclic Execution"): returns 1 if a request
+ * of `exec_time` that missed its slot still fits the current cycle after the
+ * `remaining_scheduled` time of the requests still due in it is reserved, 0 if
+ * it has to wait for the next cycle. */
+int ps_planner_outlier_fits(double cycle, double now_in_cycle, double remaining_scheduled, double exec_time);
+
 const char* ps_strerror(int status);
 /* Text of the last CUDA error seen by this service ("" if none). */
 const char* ps_last_cuda_error(ps_service* svc);

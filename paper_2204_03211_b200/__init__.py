@@ -5,4 +5,4 @@ for sm_100a under csrc/); `binding` is its ctypes face.  There is no CPU or
 library fallback: without the built .so every call raises.
 """
 from . import binding  # noqa: F401
-from .binding import Service, PsError  # noqa: F401
+from .binding import Service, Planner, PsError  # noqa: F401

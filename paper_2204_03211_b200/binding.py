@@ -78,6 +78,19 @@ _SIGNATURES = {
     "ps_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int)]),
     "ps_aggregate_block_noalloc": (C.c_int, [C.POINTER(ps_job_desc), C.c_ulonglong, C.c_size_t, C.c_void_p,
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ps_planner_create": (C.c_int, [C.POINTER(C.c_void_p), C.c_double]),
+    "ps_planner_destroy": (C.c_int, [C.c_void_p]),
+    "ps_planner_add_job": (C.c_int, [C.c_void_p, C.c_double, C.POINTER(C.c_int)]),
+    "ps_planner_assign": (C.c_int, [C.c_void_p, C.c_int, C.c_double, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
+    "ps_planner_remove_job": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int)]),
+    "ps_planner_task_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int),
+                                       C.POINTER(C.c_double)]),
+    "ps_planner_aggregator_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_double),
+                                             C.POINTER(C.c_double), C.POINTER(C.c_int)]),
+    "ps_planner_job_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                      C.POINTER(C.c_double)]),
+    "ps_planner_num_aggregators": (C.c_int, [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
+    "ps_planner_outlier_fits": (C.c_int, [C.c_double, C.c_double, C.c_double, C.c_double]),
     "ps_strerror": (C.c_char_p, [C.c_int]),
     "ps_last_cuda_error": (C.c_char_p, [C.c_void_p]),
     "ps_version": (C.c_char_p, []),
@@ -276,6 +289,69 @@ def ps_device_status(svc) -> int:
     v = C.c_int()
     _check(load().ps_device_status(svc, C.byref(v)), "ps_device_status", svc)
     return v.value
+
+
+class Planner:
+    """Thin wrapper over the ps_planner_* entry points (host-only assignment of
+    aggregation tasks to Aggregators / contexts)."""
+
+    def __init__(self, loss_limit: float = 0.1):
+        h = C.c_void_p()
+        _check(load().ps_planner_create(C.byref(h), loss_limit), "ps_planner_create")
+        self.handle = h.value
+
+    def close(self):
+        if getattr(self, "handle", None):
+            load().ps_planner_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def add_job(self, iter_duration: float) -> int:
+        j = C.c_int()
+        _check(load().ps_planner_add_job(self.handle, iter_duration, C.byref(j)), "ps_planner_add_job")
+        return j.value
+
+    def assign(self, job: int, exec_time: float):
+        t, n = C.c_int(), C.c_int()
+        _check(load().ps_planner_assign(self.handle, job, exec_time, C.byref(t), C.byref(n)), "ps_planner_assign")
+        return t.value, n.value
+
+    def remove_job(self, job: int) -> int:
+        r = C.c_int()
+        _check(load().ps_planner_remove_job(self.handle, job, C.byref(r)), "ps_planner_remove_job")
+        return r.value
+
+    def task_info(self, task: int):
+        j, n, e = C.c_int(), C.c_int(), C.c_double()
+        _check(load().ps_planner_task_info(self.handle, task, C.byref(j), C.byref(n), C.byref(e)),
+               "ps_planner_task_info")
+        return j.value, n.value, e.value
+
+    def aggregator_info(self, n: int):
+        a, c, w, k = C.c_int(), C.c_double(), C.c_double(), C.c_int()
+        _check(load().ps_planner_aggregator_info(self.handle, n, C.byref(a), C.byref(c), C.byref(w), C.byref(k)),
+               "ps_planner_aggregator_info")
+        return dict(alive=bool(a.value), cycle=c.value, load=w.value, num_tasks=k.value)
+
+    def job_info(self, job: int):
+        D, d, l = C.c_double(), C.c_double(), C.c_double()
+        _check(load().ps_planner_job_info(self.handle, job, C.byref(D), C.byref(d), C.byref(l)),
+               "ps_planner_job_info")
+        return dict(profiled=D.value, current=d.value, loss=l.value)
+
+    def num_aggregators(self):
+        a, b = C.c_int(), C.c_int()
+        _check(load().ps_planner_num_aggregators(self.handle, C.byref(a), C.byref(b)), "ps_planner_num_aggregators")
+        return a.value, b.value
+
+    @staticmethod
+    def outlier_fits(cycle, now_in_cycle, remaining_scheduled, exec_time) -> bool:
+        return bool(load().ps_planner_outlier_fits(cycle, now_in_cycle, remaining_scheduled, exec_time))
 
 
 # ---- object wrapper -----------------------------------------------------------
