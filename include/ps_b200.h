@@ -125,6 +125,24 @@ int ps_register_block(ps_service* svc, int job, int block, size_t nelem, int ctx
  * paper has one request per task per iteration), ALIGN. */
 int ps_push(ps_service* svc, int job, int block, int worker, const void* grad_dev_ptr);
 
+/* Row-sparse Push for embedding-like blocks (no counterpart in the paper, which
+ * never mentions sparsity; the result is defined as the DENSE one): the worker
+ * sends only the rows of the block it touched — `row_ids` = n_rows block-local
+ * row indices, strictly increasing (device int32 array, caller's contract, not
+ * checked), `values` = those rows packed back to back, row_len elements each, of
+ * the job's grad_dtype (device).  Rows that are not listed count as +0.0, so
+ * parameters and state come out bit-identical to pushing the dense shard with
+ * zero rows, and momentum decay / weight decay still reach every row; only the
+ * rows that exist are read.  Requirements: nelem a multiple of row_len;
+ * row_len * element size a multiple of 16 bytes; `values` 16-byte aligned (else
+ * PS_ERR_ALIGN); W <= 32.  n_rows may be 0 (both pointers still non-NULL).  A
+ * block may receive dense pushes from some workers and row-sparse ones from
+ * others, all with the same row_len within an iteration.  Launches that carry
+ * such tasks always use the direct-load kernel.
+ * Errors: BAD_ARG, ALIGN, DUPLICATE. */
+int ps_push_rows(ps_service* svc, int job, int block, int worker, const int* row_ids_dev, int n_rows,
+                 int row_len, const void* values_dev);
+
 /* n pushes in one call (host arrays of length n).  All-or-nothing. */
 int ps_push_batch(ps_service* svc, int n, const int* jobs, const int* blocks, const int* workers,
                   const void* const* grad_dev_ptrs);

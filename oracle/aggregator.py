@@ -205,6 +205,21 @@ class OracleAggregator:
             raise ValueError("bad gradient")
         b.pushed[worker] = g
 
+    def push_rows(self, job: int, block: int, worker: int, row_ids, row_len: int, values):
+        """Row-sparse push, by definition the dense push whose unlisted rows are
+        +0.0: the shard is expanded to that dense array and pushed."""
+        hp = self.jobs[job]
+        b = self.blocks[(job, block)]
+        if row_len <= 0 or b.nelem % row_len:
+            raise ValueError("block is not made of whole rows")
+        ids = np.asarray(row_ids, dtype=np.int64).reshape(-1)
+        vals = np.ascontiguousarray(values).reshape(len(ids), row_len)
+        if len(ids) and (np.any(np.diff(ids) <= 0) or ids[0] < 0 or ids[-1] >= b.nelem // row_len):
+            raise ValueError("row ids must be strictly increasing and in range")
+        dense = np.zeros((b.nelem // row_len, row_len), dtype=_grad_np_dtype(hp))   # bf16 bits 0 = +0.0
+        dense[ids] = vals
+        self.push(job, block, worker, dense.reshape(-1))
+
     def aggregate(self, ready):
         seen = set()
         for key in ready:

@@ -56,6 +56,7 @@ _SIGNATURES = {
     "ps_register_job": (C.c_int, [C.c_void_p, C.POINTER(ps_job_desc), C.POINTER(C.c_int)]),
     "ps_register_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_size_t, C.c_int, C.c_void_p]),
     "ps_push": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]),
+    "ps_push_rows": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
     "ps_push_batch": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ps_push_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
     "ps_aggregate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
@@ -169,6 +170,11 @@ def ps_register_block(svc, job: int, block: int, nelem: int, ctx: int = 0, init_
 
 def ps_push(svc, job: int, block: int, worker: int, grad):
     _check(load().ps_push(svc, job, block, worker, _ptr(grad)), "ps_push", svc)
+
+
+def ps_push_rows(svc, job: int, block: int, worker: int, row_ids, n_rows: int, row_len: int, values):
+    _check(load().ps_push_rows(svc, job, block, worker, _ptr(row_ids), n_rows, row_len, _ptr(values)),
+           "ps_push_rows", svc)
 
 
 def ps_push_batch(svc, jobs, blocks, workers, ptrs):
@@ -404,7 +410,7 @@ def _bind(name):
     return method
 
 
-for _n in ("register_job", "register_block", "push", "push_batch", "push_host", "aggregate", "pull", "pull_batch", "pull_host",
+for _n in ("register_job", "register_block", "push", "push_rows", "push_batch", "push_host", "aggregate", "pull", "pull_batch", "pull_host",
            "migrate_block", "block_stats", "block_profile", "job_profile", "block_state", "plan", "set_option", "get_option", "arena_info",
            "launch_info", "device_status"):
     setattr(Service, _n, _bind(_n))

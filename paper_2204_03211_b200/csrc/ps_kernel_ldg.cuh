@@ -5,6 +5,7 @@
 #pragma once
 
 #include "ps_math.cuh"
+#include "ps_rows.cuh"
 
 namespace psb {
 
@@ -17,12 +18,14 @@ ps_aggregate_ldg_kernel(unsigned char* __restrict__ table, const PsJobDev* __res
   PsTaskDev* tasks = reinterpret_cast<PsTaskDev*>(table + hdr->tasks_off);
   const unsigned int* starts = reinterpret_cast<const unsigned int*>(table + hdr->starts_off);
   const void* const* ptrs = reinterpret_cast<const void* const*>(table + hdr->ptrs_off);
+  const PsSparseDev* sparse = reinterpret_cast<const PsSparseDev*>(table + hdr->sparse_off);
   const unsigned int n_tasks = hdr->n_tasks, total = hdr->total_chunks;
   const bool profile = hdr->profile != 0;
 
   __shared__ unsigned int s_idx[2];
   __shared__ unsigned int s_task;
   __shared__ double s_red[kThreads / 32];
+  __shared__ const void* s_rowsrc[kThreads / 32][32];   // row-sparse tasks: a row's sources, per warp
 
   const unsigned int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   unsigned int cursor = 0;   // meaningful in warp 0
@@ -48,7 +51,11 @@ ps_aggregate_ldg_kernel(unsigned char* __restrict__ table, const PsJobDev* __res
     const size_t begin = (size_t)(idx - T->first_chunk) * chunk_elems;
     const unsigned int count = (unsigned int)min((unsigned long long)chunk_elems, T->nelem - begin);
     double sq = 0.0;
-    run_chunk_any<kThreads>(tid, jobs + T->job, T, ptrs + T->shard_row, begin, count, sq);
+    if (T->row_len)
+      run_rows_any<kThreads>(tid, jobs + T->job, T, ptrs + T->shard_row, sparse + T->sparse_row, begin, count,
+                             s_rowsrc[warp], sq);
+    else
+      run_chunk_any<kThreads>(tid, jobs + T->job, T, ptrs + T->shard_row, begin, count, sq);
 
     // chunk sum of squares: lanes, then warps, in a fixed order
 #pragma unroll

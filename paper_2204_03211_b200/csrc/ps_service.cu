@@ -45,6 +45,10 @@ struct Block {
   size_t sec = 0;                          // byte stride between p, s0, s1
   unsigned long long step = 0;
   std::vector<const void*> pushed;         // W entries, nullptr = not pushed
+  std::vector<const int*> row_ids;         // W entries, non-null = that push was row-sparse
+  std::vector<unsigned int> row_cnt;       // W entries, rows in a row-sparse push
+  unsigned int row_len = 0;                // row length of this iteration's row-sparse pushes (0 = none)
+  int nsparse = 0;
   int npushed = 0;
   unsigned int stat_idx = 0;
   unsigned long long mark = 0;             // duplicate detection inside one ready list
@@ -84,6 +88,7 @@ struct Plan {                              // one built task table (host copy)
   std::vector<unsigned char> bytes;
   std::vector<int> order;                  // block indices in table order
   unsigned int total_chunks = 0, chunk_elems = 0;
+  bool has_sparse = false;                 // some task carries row-sparse shards (direct-load kernel only)
 };
 
 }  // namespace psb
@@ -272,7 +277,14 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
   const size_t tasks_off = sizeof(PsTableHdr);
   const size_t starts_off = tasks_off + n * sizeof(PsTaskDev);
   const size_t ptrs_off = (starts_off + n * sizeof(unsigned int) + 15) / 16 * 16;
-  plan->bytes.assign(ptrs_off + nptr * sizeof(void*), 0);
+  size_t nsp = 0;                        // PsSparseDev entries: W per task that has a row-sparse push
+  for (int bi : plan->order)
+    if (s->blocks[bi].nsparse) nsp += s->jobs[s->blocks[bi].job].d.num_workers;
+  const size_t sparse_off = (ptrs_off + nptr * sizeof(void*) + 15) / 16 * 16;
+  plan->bytes.assign(sparse_off + nsp * sizeof(PsSparseDev), 0);
+  PsSparseDev* sp = reinterpret_cast<PsSparseDev*>(plan->bytes.data() + sparse_off);
+  size_t sp_row = 0;
+  plan->has_sparse = nsp > 0;
   unsigned char* base = plan->bytes.data();
   PsTaskDev* tasks = reinterpret_cast<PsTaskDev*>(base + tasks_off);
   unsigned int* starts = reinterpret_cast<unsigned int*>(base + starts_off);
@@ -290,6 +302,19 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
     t.shard_row = (unsigned int)row;
     t.first_chunk = (unsigned int)chunk;
     t.chunk_elems = ce;
+    t.row_len = 0;
+    t.sparse_row = 0;
+    if (b.nsparse) {
+      // chunks of a row-sparse task are whole rows
+      t.row_len = b.row_len;
+      t.chunk_elems = std::max(1u, ce / b.row_len) * b.row_len;
+      t.sparse_row = (unsigned int)sp_row;
+      for (int w = 0; w < j.d.num_workers; ++w) {
+        sp[sp_row + w].ids = b.row_ids[w];
+        sp[sp_row + w].n = b.row_cnt[w];
+      }
+      sp_row += j.d.num_workers;
+    }
     t.nchunks = (unsigned int)((b.nelem + t.chunk_elems - 1) / t.chunk_elems);
     t.ticket = 0;
     t.busy_ns = 0;
@@ -322,8 +347,9 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
   h->tasks_off = (unsigned int)tasks_off;
   h->starts_off = (unsigned int)starts_off;
   h->ptrs_off = (unsigned int)ptrs_off;
-  h->parts_per_chunk = use_bulk(s) ? kBulkConsumerWarps : 1;
+  h->parts_per_chunk = (use_bulk(s) && !plan->has_sparse) ? kBulkConsumerWarps : 1;
   h->profile = s->opt_profile ? 1u : 0u;
+  h->sparse_off = (unsigned int)sparse_off;
   return PS_OK;
 }
 
@@ -492,6 +518,8 @@ int ps_register_block(ps_service* s, int job, int block, size_t nelem, int ctx, 
   b.sec = Arena::round_up(nelem * sizeof(float));
   b.bytes = b.sec * (1 + j.nstate());
   b.pushed.assign(j.d.num_workers, nullptr);
+  b.row_ids.assign(j.d.num_workers, nullptr);
+  b.row_cnt.assign(j.d.num_workers, 0);
   b.stat_idx = (unsigned int)s->blocks.size();
   if (has_device(s)) PS_CUDA(s, cudaSetDevice(s->device));
   int rc = arena_alloc(s, ctx, b.bytes, &b.off);
@@ -521,6 +549,31 @@ int ps_push(ps_service* s, int job, int block, int worker, const void* ptr) {
   if (rc) return rc;
   b->pushed[worker] = ptr;
   b->npushed++;
+  return PS_OK;
+}
+
+int ps_push_rows(ps_service* s, int job, int block, int worker, const int* row_ids, int n_rows, int row_len,
+                 const void* values) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  const int bi = find_block(s, job, block);
+  if (bi < 0 || !row_ids || !values || n_rows < 0 || row_len <= 0) return PS_ERR_BAD_ARG;
+  Block& b = s->blocks[bi];
+  const Job& j = s->jobs[b.job];
+  if (worker < 0 || worker >= j.d.num_workers || j.d.num_workers > kRowsMaxWorkers) return PS_ERR_BAD_ARG;
+  if (b.nelem % (size_t)row_len != 0 || (size_t)n_rows > b.nelem / (size_t)row_len) return PS_ERR_BAD_ARG;
+  if (b.row_len != 0 && b.row_len != (unsigned int)row_len) return PS_ERR_BAD_ARG;
+  // rows are streamed with 128-bit accesses: whole vectors per row, aligned starts
+  if (((size_t)row_len * j.grad_esize()) % 16 != 0 || (reinterpret_cast<uintptr_t>(values) & 15u) ||
+      (reinterpret_cast<uintptr_t>(row_ids) & 3u))
+    return PS_ERR_ALIGN;
+  if (b.pushed[worker]) return PS_ERR_DUPLICATE;
+  b.pushed[worker] = values;
+  b.row_ids[worker] = row_ids;
+  b.row_cnt[worker] = (unsigned int)n_rows;
+  b.row_len = (unsigned int)row_len;
+  b.nsparse++;
+  b.npushed++;
   return PS_OK;
 }
 
@@ -589,7 +642,7 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
   rc = build_plan(s, idx, &plan);
   if (rc) return rc;
   Slot* sl = nullptr;
-  const bool bulk = use_bulk(s);
+  const bool bulk = use_bulk(s) && !plan.has_sparse;
   rc = acquire_slot(s, plan.bytes.size(), (size_t)plan.total_chunks * (bulk ? kBulkConsumerWarps : 1), &sl);
   if (rc) return rc;
   for (int bi : idx) {
@@ -621,6 +674,10 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
     Block& b = s->blocks[bi];
     b.step++;
     std::fill(b.pushed.begin(), b.pushed.end(), nullptr);
+    std::fill(b.row_ids.begin(), b.row_ids.end(), nullptr);
+    std::fill(b.row_cnt.begin(), b.row_cnt.end(), 0u);
+    b.row_len = 0;
+    b.nsparse = 0;
     b.npushed = 0;
     b.last_slot = slot_index;
     b.last_slot_gen = sl->gen;
@@ -970,7 +1027,8 @@ __global__ void ps_noalloc_setup_kernel(NoAllocArgs a) {
     h.ptrs_off = (unsigned int)kNaPtrsOff;
     h.parts_per_chunk = 1;
     h.profile = 0;
-    h._r0 = h._r1 = h._r2 = 0;
+    h.sparse_off = 0;
+    h._r1 = h._r2 = 0;
     *reinterpret_cast<PsTableHdr*>(base) = h;
     *reinterpret_cast<PsTaskDev*>(base + kNaTaskOff) = a.task;     // ticket = 0 inside
     *reinterpret_cast<unsigned int*>(base + kNaStartsOff) = 0;

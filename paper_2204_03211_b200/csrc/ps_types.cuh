@@ -36,8 +36,10 @@ struct __align__(16) PsTaskDev {       // 128 bytes, one per ready (job, block)
   unsigned long long step;
   unsigned int vec_ok;                 // all pointers 16-byte aligned
   unsigned int tile_elems;             // elements per ring tile (bulk-copy kernel); 0 = direct loads only
-  unsigned int chunk_elems;            // elements per chunk of THIS task (multiple of 1024)
-  unsigned int _r0, _r1, _r2;
+  unsigned int chunk_elems;            // elements per chunk of THIS task (multiple of 1024, or of row_len)
+  unsigned int row_len;                // > 0: some shards of this task are row-sparse; elements per row
+  unsigned int sparse_row;             // index of the task's first PsSparseDev entry (one per worker)
+  unsigned int _r2;
   // device-time profile of this task, filled only when the table asks for it
   unsigned long long busy_ns;          // sum over chunks of (chunk end - chunk start)      (uploaded as 0)
   unsigned long long t_first;          // earliest chunk start, %globaltimer ns             (uploaded as ~0)
@@ -53,7 +55,17 @@ struct __align__(16) PsTableHdr {      // 48 bytes at the start of the table
   unsigned int tasks_off, starts_off, ptrs_off;   // byte offsets from the table base
   unsigned int parts_per_chunk;        // partial sums each chunk publishes (1 per CTA or 1 per consumer warp)
   unsigned int profile;                // 1: record per-task device time (direct-load kernel)
-  unsigned int _r0, _r1, _r2;
+  unsigned int sparse_off;             // byte offset of the PsSparseDev array (row-sparse shards)
+  unsigned int _r1, _r2;
+};
+
+// One worker's shard of a row-sparse task: the sorted ids of the rows it holds
+// (block-local) — its values pointer sits in the ordinary shard-pointer row and
+// points at n packed rows.  ids == nullptr: this worker pushed a dense shard.
+struct __align__(16) PsSparseDev {
+  const int* ids;
+  unsigned int n;
+  unsigned int _pad;
 };
 
 struct __align__(16) PsStat {          // 48 bytes per registered block, written by the task's last chunk

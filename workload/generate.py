@@ -97,6 +97,17 @@ def grad_slab(cfg: Config, job: int, iteration: int, device="cpu", out: torch.Te
     return (out, full) if keep_fp32 else out
 
 
+def row_sparse_shards(slab: torch.Tensor, job_offset: int, nelem: int, row_len: int):
+    """The row-sparse form of one block's dense shards: per worker (row ids as
+    int32, the rows that are not entirely zero, ascending; those rows packed)."""
+    out = []
+    for w in range(slab.shape[0]):
+        rows = slab[w, job_offset:job_offset + nelem].view(-1, row_len)
+        keep = (rows != 0).any(dim=1).nonzero().squeeze(1)
+        out.append((keep.to(torch.int32).contiguous(), rows[keep].contiguous()))
+    return out
+
+
 def sample_positions(cfg: Config, job: int, per_block: int, chunk: int = 4096) -> torch.Tensor:
     """Sorted flat positions (into the job's parameter vector) to spot-check at
     full size: block starts and ends, positions around chunk boundaries, and a

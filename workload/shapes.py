@@ -129,12 +129,17 @@ MODELS = {"alexnet": alexnet, "vgg16": vgg16, "resnet50": resnet50, "awd_lm": aw
 def cut_blocks(tensors: list[Tensor], max_elems: int = BLOCK_ELEMS,
                keep_whole=lambda t: False) -> list[Block]:
     """A tensor of n elements becomes ceil(n / max_elems) blocks, all full but
-    the last; tensors for which keep_whole(t) holds stay one block."""
+    the last; tensors for which keep_whole(t) holds stay one block.  Row-sparse
+    tensors (embedding tables) are cut at row boundaries, so that a block is a
+    whole number of rows (the largest such block that fits max_elems)."""
     blocks: list[Block] = []
     job_off = 0
     for ti, t in enumerate(tensors):
         n = t.nelem
         step = n if keep_whole(t) else max_elems
+        if t.row_sparse and not keep_whole(t):
+            row_len = n // t.shape[0]
+            step = max(1, max_elems // row_len) * row_len
         off = 0
         while off < n:
             m = min(step, n - off)
