@@ -120,7 +120,7 @@ class Workload:
     """The service, the device-resident gradients and the per-round call
     arguments of one workload, prepared outside any timed region."""
 
-    def __init__(self, cfg: configs.Config, device: int, ticks: int, n_schedules: int):
+    def __init__(self, cfg: configs.Config, device: int, ticks: int, n_schedules: int, sparse: bool = False):
         from paper_2204_03211_b200 import binding as B
         self.B, self.cfg, self.device = B, cfg, device
         dev = torch.device("cuda", device)
@@ -136,26 +136,48 @@ class Workload:
             del p0
             self.slabs.append(generate.grad_slab(cfg, j, 0, dev))
         torch.cuda.synchronize(dev)
+        # row-sparse transport: blocks of embedding-like tensors are pushed as (row ids, packed rows)
+        self.sparse = {}          # (job, block) -> [(ids, values, n_rows, row_len)] per worker
+        self.sparse_saved = 0     # gradient bytes not read per step, net of the ids that are
+        if sparse:
+            for j, job in enumerate(cfg.jobs):
+                for blk in job.blocks:
+                    t = job.tensors[blk.tensor]
+                    if not t.row_sparse:
+                        continue
+                    row_len = t.nelem // t.shape[0]
+                    shards = generate.row_sparse_shards(self.slabs[j], blk.job_offset, blk.nelem, row_len)
+                    self.sparse[(j, blk.block)] = [(i, v, int(i.numel()), row_len) for i, v in shards]
+                    esz = self.slabs[j].element_size()
+                    for i, v in shards:
+                        self.sparse_saved += blk.nelem * esz - (v.numel() * esz + i.numel() * 4)
+            torch.cuda.synchronize(dev)
         # call arguments per schedule (= arrival pattern of one iteration) and round
         self.schedules = []
         for it in range(n_schedules):
             rounds = []
             for ready in configs.rounds_for(cfg, it, ticks):
                 jobs, blocks, workers, ptrs = [], [], [], []
+                rows = []
                 for (j, b) in ready:
                     job = cfg.jobs[j]
                     blk = job.blocks[b]
-                    esz = self.slabs[j].element_size()
-                    base = self.slabs[j].data_ptr()
+                    if (j, b) in self.sparse:
+                        for w, (i, v, n, rl) in enumerate(self.sparse[(j, b)]):
+                            rows.append((j, b, w, i.data_ptr(), n, rl, v.data_ptr()))
+                        continue
                     for w in range(job.num_workers):
                         jobs.append(j); blocks.append(b); workers.append(w)
                         ptrs.append(generate.shard_ptr(self.slabs[j], w, blk.job_offset))
                 rounds.append(dict(ready=ready, tasks=B.make_tasks(ready), pulled=np.empty(len(ready), np.uint64),
+                                   rows=None if not rows else tuple(
+                                       np.array([a[k] for a in rows], np.uint64 if k in (3, 6) else np.int32)
+                                       for k in range(7)),
                                    jobs=np.array(jobs, np.int32), blocks=np.array(blocks, np.int32),
                                    workers=np.array(workers, np.int32), ptrs=np.array(ptrs, np.uint64)))
             self.schedules.append(rounds)
         self.params_per_step = cfg.num_params
-        self.bytes_per_step = cfg.bytes_per_round()
+        self.bytes_per_step = cfg.bytes_per_round() - self.sparse_saved
 
     def step(self, k: int, stream) -> int:
         """Push, aggregate, pull — device-resident gradients.  Returns launches."""
@@ -163,6 +185,8 @@ class Workload:
         rounds = self.schedules[k % len(self.schedules)]
         for r in rounds:
             svc.push_batch(r["jobs"], r["blocks"], r["workers"], r["ptrs"])
+            if r["rows"] is not None:
+                svc.push_rows_batch(*r["rows"])
             svc.aggregate(r["tasks"], stream)
             svc.pull_batch(r["tasks"], r["pulled"])
         return len(rounds)
@@ -323,6 +347,9 @@ def main():
     ap.add_argument("--max-blocks", type=int, default=0, help="keep only the first N blocks of every job")
     ap.add_argument("--chunk-elems", type=int, default=0, help="PS_OPT_CHUNK_ELEMS (0 = automatic)")
     ap.add_argument("--kernel", type=int, default=0, help="PS_OPT_KERNEL (0 = automatic, 1 = direct loads, 2 = bulk-copy ring)")
+    ap.add_argument("--sparse-transport", action="store_true",
+                    help="push embedding-like blocks row-sparse (ps_push_rows); changes the bytes moved, "
+                         "so it is a separate experiment, not the default metric; implies --no-e2e")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -377,7 +404,11 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     n_sched = max(1, min(args.warmup + args.steps, 8))
-    wl = Workload(cfg, local_rank, args.ticks, n_sched)
+    wl = Workload(cfg, local_rank, args.ticks, n_sched, sparse=args.sparse_transport)
+    if args.sparse_transport:
+        args.no_e2e = True
+        config["transport"] = "row-sparse pushes for embedding tables: %.2f GB of gradient reads avoided per step" % (
+            wl.sparse_saved / 1e9)
     wl.svc.set_option(wl.B.PS_OPT_CHUNK_ELEMS, args.chunk_elems)
     wl.svc.set_option(wl.B.PS_OPT_KERNEL, args.kernel)
     stream = torch.cuda.Stream(device)

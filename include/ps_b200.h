@@ -143,6 +143,11 @@ int ps_push(ps_service* svc, int job, int block, int worker, const void* grad_de
 int ps_push_rows(ps_service* svc, int job, int block, int worker, const int* row_ids_dev, int n_rows,
                  int row_len, const void* values_dev);
 
+/* n row-sparse pushes in one call (host arrays of length n).  All-or-nothing. */
+int ps_push_rows_batch(ps_service* svc, int n, const int* jobs, const int* blocks, const int* workers,
+                       const int* const* row_ids_dev, const int* n_rows, const int* row_lens,
+                       const void* const* values_dev);
+
 /* n pushes in one call (host arrays of length n).  All-or-nothing. */
 int ps_push_batch(ps_service* svc, int n, const int* jobs, const int* blocks, const int* workers,
                   const void* const* grad_dev_ptrs);

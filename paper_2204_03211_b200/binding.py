@@ -57,6 +57,7 @@ _SIGNATURES = {
     "ps_register_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_size_t, C.c_int, C.c_void_p]),
     "ps_push": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]),
     "ps_push_rows": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
+    "ps_push_rows_batch": (C.c_int, [C.c_void_p, C.c_int] + [C.c_void_p] * 7),
     "ps_push_batch": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ps_push_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
     "ps_aggregate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
@@ -175,6 +176,13 @@ def ps_push(svc, job: int, block: int, worker: int, grad):
 def ps_push_rows(svc, job: int, block: int, worker: int, row_ids, n_rows: int, row_len: int, values):
     _check(load().ps_push_rows(svc, job, block, worker, _ptr(row_ids), n_rows, row_len, _ptr(values)),
            "ps_push_rows", svc)
+
+
+def ps_push_rows_batch(svc, jobs, blocks, workers, ids_ptrs, n_rows, row_lens, value_ptrs):
+    """int32 numpy arrays jobs/blocks/workers/n_rows/row_lens, uint64 arrays of device addresses."""
+    _check(load().ps_push_rows_batch(svc, len(jobs), jobs.ctypes.data, blocks.ctypes.data, workers.ctypes.data,
+                                     ids_ptrs.ctypes.data, n_rows.ctypes.data, row_lens.ctypes.data,
+                                     value_ptrs.ctypes.data), "ps_push_rows_batch", svc)
 
 
 def ps_push_batch(svc, jobs, blocks, workers, ptrs):
@@ -410,7 +418,7 @@ def _bind(name):
     return method
 
 
-for _n in ("register_job", "register_block", "push", "push_rows", "push_batch", "push_host", "aggregate", "pull", "pull_batch", "pull_host",
+for _n in ("register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "aggregate", "pull", "pull_batch", "pull_host",
            "migrate_block", "block_stats", "block_profile", "job_profile", "block_state", "plan", "set_option", "get_option", "arena_info",
            "launch_info", "device_status"):
     setattr(Service, _n, _bind(_n))

@@ -305,9 +305,10 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
     t.row_len = 0;
     t.sparse_row = 0;
     if (b.nsparse) {
-      // chunks of a row-sparse task are whole rows
+      // chunks of a row-sparse task are whole rows, and four times the dense size:
+      // every warp re-positions its cursors (a binary search per worker) per chunk
       t.row_len = b.row_len;
-      t.chunk_elems = std::max(1u, ce / b.row_len) * b.row_len;
+      t.chunk_elems = std::max(1u, (fixed ? ce : 4 * ce) / b.row_len) * b.row_len;
       t.sparse_row = (unsigned int)sp_row;
       for (int w = 0; w < j.d.num_workers; ++w) {
         sp[sp_row + w].ids = b.row_ids[w];
@@ -552,10 +553,44 @@ int ps_push(ps_service* s, int job, int block, int worker, const void* ptr) {
   return PS_OK;
 }
 
+static int push_rows_locked(ps_service* s, int job, int block, int worker, const int* row_ids, int n_rows,
+                            int row_len, const void* values);
+
 int ps_push_rows(ps_service* s, int job, int block, int worker, const int* row_ids, int n_rows, int row_len,
                  const void* values) {
   if (!alive(s)) return PS_ERR_BAD_HANDLE;
   std::lock_guard<std::mutex> lk(s->mu);
+  return push_rows_locked(s, job, block, worker, row_ids, n_rows, row_len, values);
+}
+
+int ps_push_rows_batch(ps_service* s, int n, const int* jobs, const int* blocks, const int* workers,
+                       const int* const* row_ids, const int* n_rows, const int* row_lens,
+                       const void* const* values) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (n < 0 || (n > 0 && (!jobs || !blocks || !workers || !row_ids || !n_rows || !row_lens || !values)))
+    return PS_ERR_BAD_ARG;
+  int rc = PS_OK, done = 0;
+  for (; done < n; ++done) {
+    rc = push_rows_locked(s, jobs[done], blocks[done], workers[done], row_ids[done], n_rows[done], row_lens[done],
+                          values[done]);
+    if (rc) break;
+  }
+  if (rc) {   // roll back: all-or-nothing
+    for (int i = 0; i < done; ++i) {
+      Block& b = s->blocks[find_block(s, jobs[i], blocks[i])];
+      b.pushed[workers[i]] = nullptr;
+      b.row_ids[workers[i]] = nullptr;
+      b.row_cnt[workers[i]] = 0;
+      b.npushed--;
+      if (--b.nsparse == 0) b.row_len = 0;
+    }
+  }
+  return rc;
+}
+
+static int push_rows_locked(ps_service* s, int job, int block, int worker, const int* row_ids, int n_rows,
+                            int row_len, const void* values) {
   const int bi = find_block(s, job, block);
   if (bi < 0 || !row_ids || !values || n_rows < 0 || row_len <= 0) return PS_ERR_BAD_ARG;
   Block& b = s->blocks[bi];
