@@ -9,7 +9,7 @@ from oracle import aggregator as A
 from paper_2204_03211_b200 import binding as B
 from workload import configs, generate
 
-TOL = 1e-6      # max |delta| <= TOL * (1 + |ref|) for fp32 state (spec tolerance; bit-equality expected)
+TOL = 1e-6      # max |delta| <= TOL * (1 + |ref|) for fp32 state (the stated tolerance; bit equality is expected and asserted too)
 
 
 def to_np(t: torch.Tensor) -> np.ndarray:
