@@ -244,7 +244,22 @@ int grid_cap(ps_service* s) {
 // rounds): 8192 elements beats 2048/4096/16384 and beats shrinking the chunks
 // toward the end of the table; the per-launch cost that remains (about 30 us)
 // is launch latency, ramp-up and the last wave, not chunk bookkeeping.
-constexpr unsigned int kChunkAuto = 8192;
+constexpr unsigned int kChunkAuto = 8192, kChunkFloor = 1024;
+
+// A launch with fewer chunks than resident CTAs leaves SMs idle while each busy
+// CTA streams a whole chunk at single-CTA bandwidth (about 19 us for 8192
+// elements, measured): such small launches get smaller chunks, halving until
+// every resident CTA has one or the floor is reached.
+unsigned int auto_chunk(ps_service* s, const std::vector<int>& idx, int grid) {
+  unsigned int ce = kChunkAuto;
+  while (ce > kChunkFloor) {
+    unsigned long long chunks = 0;
+    for (int bi : idx) chunks += (s->blocks[bi].nelem + ce - 1) / ce;
+    if (chunks >= (unsigned long long)grid) break;
+    ce >>= 1;
+  }
+  return ce;
+}
 
 // Elements per ring tile of the bulk-copy kernel: the largest multiple of 128
 // whose rows (W shards, parameters, state) fit one stage; 0 if none does.
@@ -259,7 +274,7 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
   const size_t n = idx.size();
   plan->order = idx;
   const bool fixed = s->opt_chunk > 0;
-  const unsigned int ce = fixed ? (unsigned int)s->opt_chunk : kChunkAuto;
+  const unsigned int ce = fixed ? (unsigned int)s->opt_chunk : auto_chunk(s, idx, grid_cap(s));
   plan->chunk_elems = ce;
   if (s->opt_sort) {
     // heaviest chunks first: the launch's tail is then made of light chunks

