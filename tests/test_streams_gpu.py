@@ -1,0 +1,87 @@
+"""Ordering across streams, migration failure paths, extreme worker counts."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import Pair, tiny_config, to_np
+from paper_2204_03211_b200 import binding as B
+from workload import configs, generate
+
+pytestmark = pytest.mark.gpu
+
+
+def test_same_block_on_alternating_streams_stays_ordered():
+    cfg = tiny_config([1 << 20, 70001], 4)
+    pair = Pair(cfg)
+    try:
+        streams = [torch.cuda.Stream(), torch.cuda.Stream(), None]
+        every = configs.rounds_all(cfg)[0]
+        keep = []
+        for it in range(6):
+            pair.push_iteration(it)
+            keep.append(pair.keep)                      # gradients stay alive: nothing is synchronised in the loop
+            pair.svc.aggregate(every, streams[it % 3])
+            pair.ora.aggregate(every)
+        out = torch.empty(1 << 20).pin_memory()
+        s = torch.cuda.Stream()
+        pair.svc.pull_host(0, 0, out, s)                # a fourth stream: must wait for the last aggregate
+        s.synchronize()
+        assert np.array_equal(out.numpy(), pair.ora.pull(0, 0))
+        pair.compare()
+    finally:
+        pair.close()
+
+
+def test_migration_without_room_fails_cleanly_and_block_keeps_working():
+    # blocks 0 and 2 start in context 0, block 1 in context 1 (round-robin); SGD: 2 ranges per block
+    cfg = tiny_config([200_000, 100_000, 50_000], 2)
+    cfg.num_contexts = 2
+    pair = Pair(cfg, arena_bytes=2_500_000)
+    svc = pair.svc
+    try:
+        every = configs.rounds_all(cfg)[0]
+        pair.push_iteration(0)
+        pair.aggregate(every)
+        start = [svc.arena_info(c)[0] for c in range(2)]
+        assert start == [1_600_000 + 400_384, 800_256]
+        with pytest.raises(B.PsError) as e:
+            svc.migrate_block(0, 1, 0)                  # 2,000,384 + 800,256 exceeds the arena
+        assert e.value.status == B.PS_ERR_NOMEM
+        assert svc.block_state(0, 1)[2] == 1 and [svc.arena_info(c)[0] for c in range(2)] == start
+        with pytest.raises(B.PsError) as e:
+            svc.migrate_block(0, 0, 5)
+        assert e.value.status == B.PS_ERR_BAD_ARG
+        svc.migrate_block(0, 0, 0)                      # same context: no-op
+        pair.migrate(0, 2, 1)                           # the small block fits beside block 1
+        pair.migrate(0, 2, 0)                           # and back, before the first copy was waited for
+        pair.push_iteration(1)
+        pair.aggregate(every)
+        pair.compare()
+        torch.cuda.synchronize()
+        assert [svc.arena_info(c)[0] for c in range(2)] == start
+    finally:
+        pair.close()
+
+
+@pytest.mark.parametrize("dt", [configs.F32, configs.BF16])
+def test_maximum_worker_count(dt):
+    cfg = tiny_config([4096 + 3, 9000], B.PS_MAX_WORKERS, grad_dtype=dt, grad_std=1e-3)
+    pair = Pair(cfg)
+    try:
+        for it in range(2):
+            pair.push_iteration(it)
+            pair.aggregate(configs.rounds_all(cfg)[0])
+        pair.compare()
+    finally:
+        pair.close()
+
+
+def test_destroy_with_work_in_flight_and_handle_reuse_is_rejected():
+    cfg = tiny_config([1 << 21], 8)
+    pair = Pair(cfg)
+    pair.push_iteration(0)
+    pair.svc.aggregate([(0, 0)], torch.cuda.Stream())
+    handle = pair.svc.handle
+    pair.close()                                        # waits for the launch, then frees
+    torch.cuda.synchronize()
+    assert handle is not None
