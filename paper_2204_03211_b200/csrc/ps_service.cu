@@ -33,6 +33,8 @@ constexpr unsigned int kMaxChunk = 1u << 20;
 struct Job {
   ps_job_desc d;
   std::vector<int> block_of_id;            // block id -> index into Service::blocks, -1 = none
+  mutable unsigned long long bc_step = 0;  // step the cached Adam scalars belong to
+  mutable float bc_ss = 0.f, bc_sbc2 = 0.f;
   size_t grad_esize() const { return d.grad_dtype == PS_BF16 ? 2 : 4; }
   int nstate() const { return d.opt == PS_ADAM ? 2 : 1; }
 };
@@ -337,8 +339,19 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
     t.t_first = ~0ull;
     t.t_last = 0;
     const unsigned long long step = b.step + 1;
-    t.ss_t = (float)((double)j.d.lr / (1.0 - std::pow((double)j.d.beta1, (double)step)));
-    t.sbc2_t = (float)std::sqrt(1.0 - std::pow((double)j.d.beta2, (double)step));
+    // Adam's bias-correction scalars (binary64 pow, rounded once); blocks of a job
+    // mostly share their step, so the last pair is remembered per job.  SGD: unused.
+    t.ss_t = 0.f;
+    t.sbc2_t = 0.f;
+    if (j.d.opt == PS_ADAM) {
+      if (j.bc_step != step) {
+        j.bc_step = step;
+        j.bc_ss = (float)((double)j.d.lr / (1.0 - std::pow((double)j.d.beta1, (double)step)));
+        j.bc_sbc2 = (float)std::sqrt(1.0 - std::pow((double)j.d.beta2, (double)step));
+      }
+      t.ss_t = j.bc_ss;
+      t.sbc2_t = j.bc_sbc2;
+    }
     t.job = b.job;
     t.stat_idx = b.stat_idx;
     t.step = step;
