@@ -41,12 +41,12 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from the committed ncu capture
 # (profiles/), as measured dram bytes per algorithmic byte, keyed by the hash
 # of the kernel source it was taken from.  A changed kernel reports null.
-NCU_TRAFFIC = {"kernel_sha": "fd70090e8d24", "dram_bytes_per_algorithmic_byte": 0.976}
+NCU_TRAFFIC = {"kernel_sha": "c013995b92f0", "dram_bytes_per_algorithmic_byte": 0.976}
 
 
 def kernel_sha() -> str:
     h = hashlib.sha256()
-    for name in ("ps_types.cuh", "ps_math.cuh", "ps_kernel_ldg.cuh"):
+    for name in ("ps_types.cuh", "ps_math.cuh", "ps_rows.cuh", "ps_kernel_ldg.cuh"):
         with open(os.path.join(ROOT, "paper_2204_03211_b200", "csrc", name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:12]
