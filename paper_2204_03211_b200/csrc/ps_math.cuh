@@ -139,7 +139,7 @@ __device__ __forceinline__ void chunk_bf16_vec(unsigned int tid, const Hp& h, co
     }
     float acc[8];
     widen8(ld_stream(static_cast<const unsigned short*>(ld_ptr(shards)) + e), acc);
-#pragma unroll 8
+#pragma unroll 2   // measured on B200 (W = 32): 2 beats 4, 8 and 16
     for (int w = 1; w < W; ++w) {
       float g[8];
       widen8(ld_stream(static_cast<const unsigned short*>(ld_ptr(shards, w)) + e), g);
