@@ -85,3 +85,47 @@ def test_destroy_with_work_in_flight_and_handle_reuse_is_rejected():
     pair.close()                                        # waits for the launch, then frees
     torch.cuda.synchronize()
     assert handle is not None
+
+
+def test_one_very_large_block():
+    # 2^28 + 5 elements in ONE block: 32,769 chunks, offsets beyond 2^30 bytes, a ragged tail
+    n = (1 << 28) + 5
+    cfg = tiny_config([n], 1, lr=0.05, momentum=0.5, weight_decay=1e-3)
+    pair = Pair(cfg)
+    try:
+        pair.push_iteration(0)
+        pair.aggregate([(0, 0)])
+        pair.compare()
+    finally:
+        pair.close()
+
+
+def test_concurrent_host_threads_are_serialised_by_the_service():
+    import threading
+    cfg = tiny_config([50_000] * 8, 4)
+    pair = Pair(cfg)
+    try:
+        slab = generate.grad_slab(cfg, 0, 0)
+        dslab = generate.to_device(slab, pair.dev)
+        host = to_np(slab)
+        job = cfg.jobs[0]
+        errors = []
+
+        def worker(w):
+            try:
+                for b in job.blocks:
+                    pair.svc.push(0, b.block, w, generate.shard_ptr(dslab, w, b.job_offset))
+            except Exception as e:      # noqa: BLE001
+                errors.append(e)
+
+        ts = [threading.Thread(target=worker, args=(w,)) for w in range(4)]
+        [t.start() for t in ts]
+        [t.join() for t in ts]
+        assert not errors
+        for b in job.blocks:
+            for w in range(4):
+                pair.ora.push(0, b.block, w, host[w, b.job_offset:b.job_offset + b.nelem])
+        pair.aggregate(configs.rounds_all(cfg)[0])
+        pair.compare()
+    finally:
+        pair.close()
