@@ -103,9 +103,15 @@ def load():
     """Loads libps_b200.so (built in-tree by paper_2204_03211_b200.build)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise ImportError("%s is missing: run `python -m paper_2204_03211_b200.build` "
-                              "(there is no fallback path)" % LIB_PATH)
+        # (Re)build with nvcc when the library is missing or older than its sources;
+        # if that is not possible the import fails — there is no fallback path.
+        try:
+            from . import build as _build
+            _build.build()
+        except Exception as e:      # noqa: BLE001
+            if not os.path.exists(LIB_PATH):
+                raise ImportError("%s is missing and could not be built (%s): run "
+                                  "`python -m paper_2204_03211_b200.build`" % (LIB_PATH, e))
         lib = C.CDLL(LIB_PATH)
         for name, (res, args) in _SIGNATURES.items():
             fn = getattr(lib, name)
