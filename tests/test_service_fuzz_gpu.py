@@ -35,7 +35,7 @@ def test_random_operation_sequences(seed):
     keep = []
     aggregated = 0
     try:
-        for step in range(260):
+        for step in range(400):
             op = rng.random()
             if not jobs or (op < 0.04 and len(jobs) < 6):
                 opt, dt = KINDS[int(rng.integers(4))]
@@ -115,6 +115,6 @@ def test_random_operation_sequences(seed):
                     sq, t = svc.block_stats(j, b)
                     rsq, rt = ora.block_stats(j, b)
                     assert t == rt and abs(sq - rsq) <= 1e-5 * abs(rsq) + 1e-300
-        assert aggregated > 20 and svc.device_status() == 0
+        assert aggregated >= 15 and svc.device_status() == 0
     finally:
         svc.close()
