@@ -184,6 +184,7 @@ class Workload:
                     r["c_rows"] = (len(r["rows"][0]),) + tuple(a.ctypes.data for a in r["rows"])
             self.schedules.append(rounds)
         self.lib = B.load()
+        self.overlap = False
         self.params_per_step = cfg.num_params
         self.bytes_per_step = cfg.bytes_per_round() - self.sparse_saved
 
@@ -203,6 +204,8 @@ class Workload:
                 rc = lib.ps_pull_batch(h, r["tasks"], r["n"], r["c_pulled"])
             if rc:
                 raise self.B.PsError(rc, "bench step")
+        if self.overlap:
+            lib.ps_join(h, sp)      # the step's launches overlapped each other; the stream joins them here
         return len(rounds)
 
     # ---- end to end: host gradients in, host parameters out
@@ -364,6 +367,9 @@ def main():
     ap.add_argument("--sparse-transport", action="store_true",
                     help="push embedding-like blocks row-sparse (ps_push_rows); changes the bytes moved, "
                          "so it is a separate experiment, not the default metric; implies --no-e2e")
+    ap.add_argument("--in-stream", action="store_true",
+                    help="enqueue every launch on the caller's stream (PS_OPT_OVERLAP = 0) instead of letting "
+                         "the launches of a step overlap on the service's streams and joining once per step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -425,6 +431,9 @@ def main():
             wl.sparse_saved / 1e9)
     wl.svc.set_option(wl.B.PS_OPT_CHUNK_ELEMS, args.chunk_elems)
     wl.svc.set_option(wl.B.PS_OPT_KERNEL, args.kernel)
+    wl.overlap = not args.in_stream
+    wl.svc.set_option(wl.B.PS_OPT_OVERLAP, int(wl.overlap))
+    config["launch_mode"] = "overlapped, one ps_join per step" if wl.overlap else "in-stream"
     stream = torch.cuda.Stream(device)
 
     for k in range(args.warmup):

@@ -79,6 +79,15 @@ enum {
                               Must be a multiple of 1024 (<= 2^20) when non-zero. */
   PS_OPT_CTAS_PER_SM = 2,  /* persistent CTAs per SM; 0 = automatic */
   PS_OPT_SORT_TASKS = 3,   /* 1 (default): heaviest chunks first inside a launch; 0: caller's order */
+  PS_OPT_OVERLAP = 6,      /* 1: ps_aggregate runs its launch on service-owned streams, ordered after
+                              the work enqueued on `stream` at call time and after earlier launches
+                              that touch the same blocks, but NOT joined back into `stream`:
+                              consecutive launches overlap (the tail of one with the head of the
+                              next).  The caller joins with ps_join(svc, stream) before it reuses
+                              gradient buffers or reads results on its own streams; ps_pull_host,
+                              ps_block_stats, ps_block_profile, ps_migrate_block and ps_push_host
+                              order themselves after the block's last launch in either mode.
+                              Default 0: every launch is enqueued on `stream` itself. */
   PS_OPT_PROFILE = 5,      /* 1: aggregates record per-task device time (see ps_block_profile);
                               costs a few atomics per chunk; direct-load kernel only; default 0 */
   PS_OPT_KERNEL = 4        /* kernel variant: 0 = automatic (direct loads), 1 = direct loads,
@@ -172,6 +181,10 @@ int ps_push_host(ps_service* svc, int job, int block, int worker, const void* gr
  * Errors (nothing launched, nothing changed): BAD_ARG, DUPLICATE, NOT_READY,
  * NO_DEVICE, NOMEM, CUDA. */
 int ps_aggregate(ps_service* svc, const ps_task* ready, int n_ready, void* stream);
+
+/* Makes `stream` wait for every ps_aggregate launch enqueued so far that it has
+ * not joined yet (needed only with PS_OPT_OVERLAP; otherwise a no-op). */
+int ps_join(ps_service* svc, void* stream);
 
 /* Pull (paper Section 4): *params_dev_ptr_out receives a device pointer to the
  * block's nelem fp32 parameters.  Borrowed; stable until the block is migrated

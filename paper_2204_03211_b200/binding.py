@@ -24,6 +24,7 @@ PS_NOALLOC_MAX_ELEMS = 1 << 24
 PS_DEVICE_NONE = -1
 PS_MAX_WORKERS = 256
 PS_OPT_CHUNK_ELEMS, PS_OPT_CTAS_PER_SM, PS_OPT_SORT_TASKS, PS_OPT_KERNEL, PS_OPT_PROFILE = 1, 2, 3, 4, 5
+PS_OPT_OVERLAP = 6
 
 
 class ps_job_desc(C.Structure):
@@ -61,6 +62,7 @@ _SIGNATURES = {
     "ps_push_batch": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ps_push_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
     "ps_aggregate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
+    "ps_join": (C.c_int, [C.c_void_p, C.c_void_p]),
     "ps_pull": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p)]),
     "ps_pull_batch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "ps_pull_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
@@ -213,6 +215,10 @@ def make_tasks(pairs):
 def ps_aggregate(svc, ready, stream=None):
     tasks = ready if isinstance(ready, C.Array) else make_tasks(list(ready))
     _check(load().ps_aggregate(svc, tasks, len(tasks), _stream_ptr(stream)), "ps_aggregate", svc)
+
+
+def ps_join(svc, stream=None):
+    _check(load().ps_join(svc, _stream_ptr(stream)), "ps_join", svc)
 
 
 def ps_pull(svc, job: int, block: int) -> int:
@@ -424,7 +430,7 @@ def _bind(name):
     return method
 
 
-for _n in ("register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "aggregate", "pull", "pull_batch", "pull_host",
+for _n in ("register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "aggregate", "join", "pull", "pull_batch", "pull_host",
            "migrate_block", "block_stats", "block_profile", "job_profile", "block_state", "plan", "set_option", "get_option", "arena_info",
            "launch_info", "device_status"):
     setattr(Service, _n, _bind(_n))

@@ -82,6 +82,7 @@ struct Slot {
   size_t partial_cap = 0;
   cudaEvent_t done = nullptr;
   cudaEvent_t copied = nullptr;            // table upload finished (recorded on the copy stream)
+  cudaEvent_t input = nullptr;             // overlap mode: the caller's stream at the time of the call
   bool inflight = false;
   unsigned long long gen = 0;
 };
@@ -116,6 +117,10 @@ struct ps_service {
   long long opt_chunk = 0, opt_ctas = 0, opt_sort = 1, opt_kernel = 0, opt_profile = 0;
   int* status_dev = nullptr;               // error word written by kernels whose waits expired
   cudaStream_t copy_stream = nullptr;      // table uploads run here, beside the previous launch
+  cudaStream_t work_streams[2] = {nullptr, nullptr};   // overlap mode: launches alternate between these
+  int next_work = 0;
+  unsigned int unjoined = 0;               // overlap mode: slots whose launch no caller stream has joined yet
+  long long opt_overlap = 0;
   int occ_ctas = 0;
   unsigned long long launches = 0;
   int last_grid = 0, last_block = 0;
@@ -390,6 +395,8 @@ int acquire_slot(ps_service* s, size_t table_bytes, size_t nchunks, Slot** out) 
   }
   if (!sl.done) PS_CUDA(s, cudaEventCreateWithFlags(&sl.done, cudaEventDisableTiming));
   if (!sl.copied) PS_CUDA(s, cudaEventCreateWithFlags(&sl.copied, cudaEventDisableTiming));
+  if (!sl.input) PS_CUDA(s, cudaEventCreateWithFlags(&sl.input, cudaEventDisableTiming));
+  s->unjoined &= ~(1u << (unsigned)(&sl - s->slots));   // its previous launch has completed (host waited)
   if (table_bytes > sl.cap) {
     size_t ncap = std::max<size_t>(table_bytes * 2, 1 << 16);
     if (sl.host) PS_CUDA(s, cudaFreeHost(sl.host));
@@ -412,10 +419,16 @@ int acquire_slot(ps_service* s, size_t table_bytes, size_t nchunks, Slot** out) 
 }
 
 // Makes `stream` wait for everything enqueued so far that touches block b.
-int order_after_block(ps_service* s, Block& b, cudaStream_t stream) {
+// `waited` (optional) collects the slots this call has already made `stream`
+// wait for, so that a list of many blocks from one earlier launch costs one wait.
+int order_after_block(ps_service* s, Block& b, cudaStream_t stream, unsigned int* waited = nullptr) {
   if (b.last_slot >= 0) {
     Slot& sl = s->slots[b.last_slot];
-    if (sl.inflight && sl.gen == b.last_slot_gen) PS_CUDA(s, cudaStreamWaitEvent(stream, sl.done, 0));
+    const unsigned int bit = 1u << (unsigned)b.last_slot;
+    if (sl.inflight && sl.gen == b.last_slot_gen && !(waited && (*waited & bit))) {
+      PS_CUDA(s, cudaStreamWaitEvent(stream, sl.done, 0));
+      if (waited) *waited |= bit;
+    }
   }
   if (b.mig_pending) {
     cudaError_t q = cudaEventQuery(b.mig_event);
@@ -458,6 +471,8 @@ int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(ps_aggregate_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBulkSmemBytes);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i)
+      e = cudaStreamCreateWithFlags(&s->work_streams[i], cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaMalloc(&s->status_dev, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(s->status_dev, 0, sizeof(int));
     for (int c = 0; e == cudaSuccess && c < num_contexts; ++c) {
@@ -470,6 +485,7 @@ int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes
       for (auto& c : s->ctxs) if (c.base) cudaFree(c.base);
       if (s->status_dev) cudaFree(s->status_dev);
       if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
+      for (auto ws : s->work_streams) if (ws) cudaStreamDestroy(ws);
       cudaGetLastError();
       delete s;
       return oom ? PS_ERR_NOMEM : PS_ERR_CUDA;
@@ -494,12 +510,14 @@ int ps_destroy(ps_service* s) {
       if (sl.partials) cudaFree(sl.partials);
       if (sl.done) cudaEventDestroy(sl.done);
       if (sl.copied) cudaEventDestroy(sl.copied);
+      if (sl.input) cudaEventDestroy(sl.input);
     }
     for (auto& c : s->ctxs) if (c.base) cudaFree(c.base);
     if (s->jobs_dev) cudaFree(s->jobs_dev);
     if (s->stats_dev) cudaFree(s->stats_dev);
     if (s->status_dev) cudaFree(s->status_dev);
     if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
+    for (auto ws : s->work_streams) if (ws) cudaStreamDestroy(ws);
   }
   s->magic = 0;
   delete s;
@@ -683,6 +701,9 @@ int ps_push_host(ps_service* s, int job, int block, int worker, const void* host
       return PS_ERR_CUDA;
     }
   }
+  // the staging buffer may still be read by the block's previous aggregate
+  rc = order_after_block(s, *b, static_cast<cudaStream_t>(stream));
+  if (rc) return rc;
   char* dst = static_cast<char*>(b->staging) + (size_t)worker * b->staging_row;
   PS_CUDA(s, cudaMemcpyAsync(dst, host_ptr, b->nelem * j.grad_esize(), cudaMemcpyHostToDevice,
                              static_cast<cudaStream_t>(stream)));
@@ -708,8 +729,20 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
   const bool bulk = use_bulk(s) && !plan.has_sparse;
   rc = acquire_slot(s, plan.bytes.size(), (size_t)plan.total_chunks * (bulk ? kBulkConsumerWarps : 1), &sl);
   if (rc) return rc;
+  const int slot_index = (int)(sl - s->slots);
+  // Overlap mode: the launch goes to one of two service-owned streams, after the
+  // work the caller has enqueued on `stream` so far; consecutive launches then
+  // overlap (the next one's CTAs fill the SMs the previous one's tail leaves idle).
+  cudaStream_t run = stream;
+  if (s->opt_overlap) {
+    run = s->work_streams[s->next_work];
+    s->next_work ^= 1;
+    PS_CUDA(s, cudaEventRecord(sl->input, stream));
+    PS_CUDA(s, cudaStreamWaitEvent(run, sl->input, 0));
+  }
+  unsigned int waited = 0;
   for (int bi : idx) {
-    rc = order_after_block(s, s->blocks[bi], stream);
+    rc = order_after_block(s, s->blocks[bi], run, &waited);
     if (rc) return rc;
   }
   std::memcpy(sl->host, plan.bytes.data(), plan.bytes.size());
@@ -717,17 +750,17 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
   // service's own stream and overlaps the previous launch; the kernel waits for it.
   PS_CUDA(s, cudaMemcpyAsync(sl->dev, sl->host, plan.bytes.size(), cudaMemcpyHostToDevice, s->copy_stream));
   PS_CUDA(s, cudaEventRecord(sl->copied, s->copy_stream));
-  PS_CUDA(s, cudaStreamWaitEvent(stream, sl->copied, 0));
+  PS_CUDA(s, cudaStreamWaitEvent(run, sl->copied, 0));
   const int grid = (int)std::min<unsigned long long>(plan.total_chunks, (unsigned long long)grid_cap(s));
   if (bulk)
-    ps_aggregate_bulk_kernel<<<grid, kBulkThreads, kBulkSmemBytes, stream>>>(sl->dev, s->jobs_dev, s->stats_dev,
-                                                                             sl->partials, s->status_dev);
+    ps_aggregate_bulk_kernel<<<grid, kBulkThreads, kBulkSmemBytes, run>>>(sl->dev, s->jobs_dev, s->stats_dev,
+                                                                          sl->partials, s->status_dev);
   else
-    ps_aggregate_ldg_kernel<<<grid, kThreads, 0, stream>>>(sl->dev, s->jobs_dev, s->stats_dev, sl->partials);
+    ps_aggregate_ldg_kernel<<<grid, kThreads, 0, run>>>(sl->dev, s->jobs_dev, s->stats_dev, sl->partials);
   PS_CUDA(s, cudaGetLastError());
-  PS_CUDA(s, cudaEventRecord(sl->done, stream));
+  PS_CUDA(s, cudaEventRecord(sl->done, run));
   sl->inflight = true;
-  const int slot_index = (int)(sl - s->slots);
+  if (s->opt_overlap) s->unjoined |= 1u << (unsigned)slot_index;
   s->next_slot = (s->next_slot + 1) % kSlots;
   s->launches++;
   s->last_grid = grid;
@@ -745,6 +778,20 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
     b.last_slot = slot_index;
     b.last_slot_gen = sl->gen;
   }
+  return PS_OK;
+}
+
+int ps_join(ps_service* s, void* stream_) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (!has_device(s)) return PS_OK;
+  PS_CUDA(s, cudaSetDevice(s->device));
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  for (int i = 0; i < kSlots; ++i) {
+    if (!(s->unjoined & (1u << i))) continue;
+    if (s->slots[i].inflight) PS_CUDA(s, cudaStreamWaitEvent(stream, s->slots[i].done, 0));
+  }
+  s->unjoined = 0;
   return PS_OK;
 }
 
@@ -961,6 +1008,9 @@ int ps_set_option(ps_service* s, int option, long long value) {
     case PS_OPT_PROFILE:
       s->opt_profile = value ? 1 : 0;
       return PS_OK;
+    case PS_OPT_OVERLAP:
+      s->opt_overlap = value ? 1 : 0;
+      return PS_OK;
     default:
       return PS_ERR_BAD_ARG;
   }
@@ -976,6 +1026,7 @@ int ps_get_option(ps_service* s, int option, long long* out) {
     case PS_OPT_SORT_TASKS: *out = s->opt_sort; return PS_OK;
     case PS_OPT_KERNEL: *out = s->opt_kernel; return PS_OK;
     case PS_OPT_PROFILE: *out = s->opt_profile; return PS_OK;
+    case PS_OPT_OVERLAP: *out = s->opt_overlap; return PS_OK;
     default: return PS_ERR_BAD_ARG;
   }
 }

@@ -57,20 +57,25 @@ def test_c3_vgg16_shaped_20_iterations():
         pair.close()
 
 
-def test_c4_twelve_packed_jobs_bursty_arrival():
+@pytest.mark.parametrize("overlap", [0, 1], ids=["in-stream", "overlapped"])
+def test_c4_twelve_packed_jobs_bursty_arrival(overlap):
+    from paper_2204_03211_b200 import binding as B
     cfg = configs.c4()
     pair = SampledPair(cfg, per_block=128, full_per_job=4)
     try:
+        pair.svc.set_option(B.PS_OPT_OVERLAP, overlap)      # the launch configuration bench.py times is "overlapped"
         stream = torch.cuda.Stream()
         for it in range(cfg.iterations):
             rounds = configs.rounds_for(cfg, it, 16)
             assert all(len({j for j, _ in r}) >= 1 for r in rounds)
             pair.iteration(it, rounds, stream)
+            pair.svc.join(stream)
             stream.synchronize()
         pair.compare(cfg.iterations)
         # one more iteration with everything ready at once: a single packed launch
         before = pair.svc.launch_info()["launches"]
         pair.iteration(cfg.iterations, configs.rounds_all(cfg), stream)
+        pair.svc.join(stream)
         stream.synchronize()
         assert pair.svc.launch_info()["launches"] == before + 1
         pair.compare(cfg.iterations + 1)

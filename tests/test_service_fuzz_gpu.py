@@ -24,11 +24,12 @@ def _status(fn, *a):
     return 0
 
 
-@pytest.mark.parametrize("seed", [0, 1, 2])
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
 def test_random_operation_sequences(seed):
     rng = np.random.default_rng(seed)
     nctx = 3
     svc = B.Service(0, nctx, 64 << 20)
+    svc.set_option(B.PS_OPT_OVERLAP, seed % 2)          # odd seeds: launches on the service's own streams
     ora = A.OracleAggregator(nctx)
     streams = [None, torch.cuda.Stream(), torch.cuda.Stream()]
     jobs, blocks = [], {}            # blocks[(j, b)] = dict(n, rows, pushed=set)
