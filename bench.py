@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from the committed ncu capture
 # (profiles/), as measured dram bytes per algorithmic byte, keyed by the hash
 # of the kernel source it was taken from.  A changed kernel reports null.
-NCU_TRAFFIC = {"kernel_sha": "c013995b92f0", "dram_bytes_per_algorithmic_byte": 0.976}
+NCU_TRAFFIC = {"kernel_sha": "46c48da750e1", "dram_bytes_per_algorithmic_byte": 0.976}
 
 
 def kernel_sha() -> str:
@@ -484,7 +484,7 @@ def main():
                          "frac_of_nominal_8TBs": achieved / 8000.0, "kernel": info["kernel"],
                          "bytes_per_launch": per_launch_bytes, "kernel_sha": sha,
                          "note": "duration = event time of the whole timed region / launches "
-                                 "(includes the per-launch table upload)"},
+                                 "(launches of a step may overlap; table uploads included)"},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
             "launch": {"grid": info["grid"], "block": info["block"]},
             "host_ms_per_step": host_ms / args.steps, "clocks": clocks,
