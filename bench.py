@@ -226,6 +226,8 @@ class Workload:
             off += n
         self.out = torch.empty(self.cfg.num_params, dtype=torch.float32).pin_memory()
         self.pool_bytes = pool_bytes
+        self.pull_stream = torch.cuda.Stream(torch.device("cuda", self.device))
+        self.pull_done = torch.cuda.Event()
         self.h2d = total
         self.d2h = self.cfg.num_params * 4
 
@@ -250,8 +252,14 @@ class Workload:
                     svc.push_host(j, b, w, pool_ptr + cursor, stream)
                     cursor += (nbytes + 255) // 256 * 256
             svc.aggregate(r["tasks"], stream)
+            # parameters travel back on a second stream (the library orders each copy after the
+            # block's aggregate), so device-to-host traffic overlaps the next round's uploads
             for (j, b) in r["ready"]:
-                svc.pull_host(j, b, out_ptr + 4 * (out_off[j] + cfg.jobs[j].blocks[b].job_offset), stream)
+                svc.pull_host(j, b, out_ptr + 4 * (out_off[j] + cfg.jobs[j].blocks[b].job_offset), self.pull_stream)
+        self.pull_done.record(self.pull_stream)
+        stream.wait_event(self.pull_done)           # the step ends when its last result is on the host
+        if self.overlap:
+            svc.join(stream)
         return len(rounds)
 
 
