@@ -210,6 +210,15 @@ int ps_pull_host(ps_service* svc, int job, int block, float* params_host_dst, vo
  * Errors: BAD_ARG, NOMEM (block stays where it was), NO_DEVICE, CUDA. */
 int ps_migrate_block(ps_service* svc, int job, int block, int dst_ctx, void* stream);
 
+/* The same for n blocks at once (host array of tasks, no block listed twice), as
+ * ONE batch: every destination range is reserved first (PS_ERR_NOMEM leaves all
+ * blocks where they were), one gather-copy kernel per 96 blocks moves the data
+ * and one event marks the batch — moving all tensors of a model costs a few
+ * launches instead of one copy call per tensor (the paper's Appendix B measures
+ * exactly that case: the overhead of migrating all tensors of a model).
+ * Errors: BAD_ARG, DUPLICATE, NOMEM, NO_DEVICE, CUDA. */
+int ps_migrate_blocks(ps_service* svc, const ps_task* tasks, int n, int dst_ctx, void* stream);
+
 /* Per-block statistics of the last aggregate (paper Section 3.1: profilers feed
  * the manager): squared norm of the aggregated gradient and the step counter.
  * Waits for the block's last aggregate to finish.  Either out pointer may be

@@ -66,6 +66,7 @@ _SIGNATURES = {
     "ps_pull": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p)]),
     "ps_pull_batch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "ps_pull_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
+    "ps_migrate_blocks": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]),
     "ps_migrate_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]),
     "ps_block_stats": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_ulonglong)]),
     "ps_block_profile": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double)]),
@@ -243,6 +244,11 @@ def ps_pull_host(svc, job: int, block: int, dst_host, stream=None):
 
 def ps_migrate_block(svc, job: int, block: int, dst_ctx: int, stream=None):
     _check(load().ps_migrate_block(svc, job, block, dst_ctx, _stream_ptr(stream)), "ps_migrate_block", svc)
+
+
+def ps_migrate_blocks(svc, tasks, dst_ctx: int, stream=None):
+    t = tasks if isinstance(tasks, C.Array) else make_tasks(list(tasks))
+    _check(load().ps_migrate_blocks(svc, t, len(t), dst_ctx, _stream_ptr(stream)), "ps_migrate_blocks", svc)
 
 
 def ps_block_stats(svc, job: int, block: int):
@@ -431,6 +437,6 @@ def _bind(name):
 
 
 for _n in ("register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "aggregate", "join", "pull", "pull_batch", "pull_host",
-           "migrate_block", "block_stats", "block_profile", "job_profile", "block_state", "plan", "set_option", "get_option", "arena_info",
+           "migrate_block", "migrate_blocks", "block_stats", "block_profile", "job_profile", "block_state", "plan", "set_option", "get_option", "arena_info",
            "launch_info", "device_status"):
     setattr(Service, _n, _bind(_n))

@@ -5,3 +5,4 @@
 #include "ps_math.cuh"
 #include "ps_kernel_ldg.cuh"
 #include "ps_kernel_bulk.cuh"
+#include "ps_migrate.cuh"

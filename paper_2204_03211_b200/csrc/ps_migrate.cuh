@@ -1,0 +1,41 @@
+// Gather-copy kernel of block migration: moves up to kMigPerLaunch (source,
+// destination, bytes) ranges between context arenas in ONE launch (paper Section
+// 3.2 and Appendix B: the old Aggregator copies the tensor's contents — parameters
+// and metadata, here the optimizer state — to the new one).  Ranges are 256-byte
+// aligned and a multiple of 256 bytes long (arena granularity); work is cut
+// into 64 KB tiles that CTAs take round-robin.
+#pragma once
+
+#include <cuda_runtime.h>
+
+namespace psb {
+
+constexpr int kMigPerLaunch = 96;
+constexpr unsigned int kMigTile = 65536;
+
+struct MigArgs {                       // passed by value (about 2.7 KB of kernel parameters)
+  const unsigned char* src[kMigPerLaunch];
+  unsigned char* dst[kMigPerLaunch];
+  unsigned long long bytes[kMigPerLaunch];
+  unsigned int tile_prefix[kMigPerLaunch + 1];   // first tile of each range; [n] = total tiles
+  int n;
+};
+
+__global__ void __launch_bounds__(256) ps_migrate_kernel(const MigArgs a) {
+  const unsigned int total = a.tile_prefix[a.n];
+  for (unsigned int t = blockIdx.x; t < total; t += gridDim.x) {
+    int lo = 0, hi = a.n;                          // largest d with tile_prefix[d] <= t
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (a.tile_prefix[mid] <= t) lo = mid; else hi = mid;
+    }
+    const unsigned long long off = (unsigned long long)(t - a.tile_prefix[lo]) * kMigTile;
+    const unsigned long long left = a.bytes[lo] - off;
+    const unsigned int len = left < kMigTile ? (unsigned int)left : kMigTile;
+    const uint4* s = reinterpret_cast<const uint4*>(a.src[lo] + off);
+    uint4* d = reinterpret_cast<uint4*>(a.dst[lo] + off);
+    for (unsigned int i = threadIdx.x; i < len / 16; i += 256) d[i] = __ldcs(s + i);
+  }
+}
+
+}  // namespace psb

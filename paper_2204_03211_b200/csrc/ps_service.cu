@@ -56,8 +56,7 @@ struct Block {
   unsigned long long mark = 0;             // duplicate detection inside one ready list
   int last_slot = -1;                      // slot of the last aggregate
   unsigned long long last_slot_gen = 0;
-  cudaEvent_t mig_event = nullptr;
-  bool mig_pending = false;
+  int mig_batch = -1;                      // migration batch whose copy may still be in flight
   void* staging = nullptr;                 // device buffer for ps_push_host
   size_t staging_row = 0;
 };
@@ -67,11 +66,20 @@ struct Ctx {
   Arena arena;
 };
 
-struct PendingFree {
+struct PendingFree {                       // source range of a migration, released when its batch has landed
   int ctx;
   size_t off, bytes;
-  cudaEvent_t ev;                          // owned by the block; only queried here
-  int block;
+  int batch;
+};
+
+// One ps_migrate_block(s) call: its copies complete together, at `ev`.
+struct MigBatch {
+  cudaEvent_t ev = nullptr;
+  bool pending = false;
+  unsigned long long seen_call = 0;        // the event was last queried during this API call ...
+  bool seen_ready = false;                 // ... with this answer
+  unsigned long long waited_call = 0;      // a stream wait was issued during this API call ...
+  cudaStream_t waited_stream = nullptr;    // ... on this stream
 };
 
 struct Slot {
@@ -107,6 +115,8 @@ struct ps_service {
   std::vector<Job> jobs;
   std::vector<Block> blocks;
   std::vector<PendingFree> pending_free;
+  std::vector<MigBatch> batches;
+  unsigned long long call_id = 0;          // counts API calls that order work (dedupes event queries/waits)
   PsJobDev* jobs_dev = nullptr;
   size_t jobs_dev_cap = 0;
   PsStat* stats_dev = nullptr;
@@ -157,19 +167,35 @@ float* blk_s1(ps_service* s, const Block& b) {
 
 // Releases source ranges of finished migrations.  With wait = true blocks
 // until every pending copy has completed.
+// Has the batch's copy landed?  The event is queried at most once per API call.
+// *ready_out = false also when the query itself failed (rc != PS_OK).
+int batch_ready(ps_service* s, int batch, bool wait, bool* ready_out) {
+  MigBatch& m = s->batches[batch];
+  *ready_out = true;
+  if (!m.pending) return PS_OK;
+  if (!wait && m.seen_call == s->call_id) { *ready_out = m.seen_ready; return PS_OK; }
+  cudaError_t q = wait ? cudaEventSynchronize(m.ev) : cudaEventQuery(m.ev);
+  if (q != cudaSuccess && q != cudaErrorNotReady) {
+    *ready_out = false;
+    s->cuda_err = std::string("migration event: ") + cudaGetErrorString(q);
+    return PS_ERR_CUDA;
+  }
+  m.seen_call = s->call_id;
+  m.seen_ready = (q == cudaSuccess);
+  if (m.seen_ready) m.pending = false;
+  *ready_out = m.seen_ready;
+  return PS_OK;
+}
+
 int reap_frees(ps_service* s, bool wait) {
   size_t keep = 0;
   for (size_t i = 0; i < s->pending_free.size(); ++i) {
     PendingFree& f = s->pending_free[i];
-    cudaError_t q = wait ? cudaEventSynchronize(f.ev) : cudaEventQuery(f.ev);
-    if (q == cudaSuccess) {
-      s->ctxs[f.ctx].arena.release(f.off, f.bytes);
-    } else if (q == cudaErrorNotReady) {
-      s->pending_free[keep++] = f;
-    } else {
-      s->cuda_err = std::string("migration event: ") + cudaGetErrorString(q);
-      return PS_ERR_CUDA;
-    }
+    bool ready = false;
+    int rc = batch_ready(s, f.batch, wait, &ready);
+    if (rc) return rc;
+    if (ready) s->ctxs[f.ctx].arena.release(f.off, f.bytes);
+    else s->pending_free[keep++] = f;
   }
   s->pending_free.resize(keep);
   return PS_OK;
@@ -430,11 +456,20 @@ int order_after_block(ps_service* s, Block& b, cudaStream_t stream, unsigned int
       if (waited) *waited |= bit;
     }
   }
-  if (b.mig_pending) {
-    cudaError_t q = cudaEventQuery(b.mig_event);
-    if (q == cudaSuccess) b.mig_pending = false;
-    else if (q == cudaErrorNotReady) PS_CUDA(s, cudaStreamWaitEvent(stream, b.mig_event, 0));
-    else { s->cuda_err = cudaGetErrorString(q); return PS_ERR_CUDA; }
+  if (b.mig_batch >= 0) {
+    bool ready = false;
+    int rc = batch_ready(s, b.mig_batch, false, &ready);
+    if (rc) return rc;
+    if (ready) {
+      b.mig_batch = -1;
+    } else {
+      MigBatch& m = s->batches[b.mig_batch];
+      if (!(m.waited_call == s->call_id && m.waited_stream == stream)) {
+        PS_CUDA(s, cudaStreamWaitEvent(stream, m.ev, 0));
+        m.waited_call = s->call_id;
+        m.waited_stream = stream;
+      }
+    }
   }
   return PS_OK;
 }
@@ -500,10 +535,10 @@ int ps_destroy(ps_service* s) {
   if (has_device(s)) {
     cudaSetDevice(s->device);
     cudaDeviceSynchronize();
-    for (auto& b : s->blocks) {
-      if (b.mig_event) cudaEventDestroy(b.mig_event);
+    for (auto& b : s->blocks)
       if (b.staging) cudaFree(b.staging);
-    }
+    for (auto& m : s->batches)
+      if (m.ev) cudaEventDestroy(m.ev);
     for (auto& sl : s->slots) {
       if (sl.host) cudaFreeHost(sl.host);
       if (sl.dev) cudaFree(sl.dev);
@@ -702,6 +737,7 @@ int ps_push_host(ps_service* s, int job, int block, int worker, const void* host
     }
   }
   // the staging buffer may still be read by the block's previous aggregate
+  ++s->call_id;
   rc = order_after_block(s, *b, static_cast<cudaStream_t>(stream));
   if (rc) return rc;
   char* dst = static_cast<char*>(b->staging) + (size_t)worker * b->staging_row;
@@ -722,6 +758,7 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
   if (idx.empty()) return PS_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   PS_CUDA(s, cudaSetDevice(s->device));
+  ++s->call_id;
   Plan plan;
   rc = build_plan(s, idx, &plan);
   if (rc) return rc;
@@ -857,9 +894,89 @@ int ps_pull_host(ps_service* s, int job, int block, float* dst, void* stream_) {
   PS_CUDA(s, cudaSetDevice(s->device));
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   Block& b = s->blocks[bi];
+  ++s->call_id;
   int rc = order_after_block(s, b, stream);
   if (rc) return rc;
   PS_CUDA(s, cudaMemcpyAsync(dst, blk_p(s, b), b.nelem * sizeof(float), cudaMemcpyDeviceToHost, stream));
+  return PS_OK;
+}
+
+// Moves the listed blocks (indices into s->blocks) to dst_ctx as ONE batch: all
+// destination ranges are reserved first (nothing changes if one does not fit),
+// the copies are ordered after each block's last aggregate and last move, one
+// gather-copy kernel per 96 blocks (a plain cudaMemcpyAsync for a single block)
+// does the transfer, and one event marks the whole batch.
+static int migrate_many(ps_service* s, const std::vector<int>& bis, int dst_ctx, cudaStream_t stream) {
+  struct Move { int bi; size_t noff; };
+  std::vector<Move> moves;
+  for (int bi : bis) {
+    Block& b = s->blocks[bi];
+    if (b.ctx == dst_ctx) continue;
+    size_t noff = 0;
+    int rc = arena_alloc(s, dst_ctx, b.bytes, &noff);
+    if (rc) {
+      for (auto& m : moves) s->ctxs[dst_ctx].arena.release(m.noff, s->blocks[m.bi].bytes);
+      return rc;
+    }
+    moves.push_back(Move{bi, noff});
+  }
+  if (moves.empty()) return PS_OK;
+  auto undo = [&]() {
+    for (auto& m : moves) s->ctxs[dst_ctx].arena.release(m.noff, s->blocks[m.bi].bytes);
+  };
+  int batch = -1;
+  for (int i = 0; i < (int)s->batches.size(); ++i)
+    if (!s->batches[i].pending) { batch = i; break; }
+  if (batch < 0) {
+    s->batches.emplace_back();
+    batch = (int)s->batches.size() - 1;
+  }
+  if (!s->batches[batch].ev) {
+    cudaError_t e = cudaEventCreateWithFlags(&s->batches[batch].ev, cudaEventDisableTiming);
+    if (e != cudaSuccess) { undo(); s->cuda_err = cudaGetErrorString(e); return PS_ERR_CUDA; }
+  }
+  unsigned int waited = 0;
+  for (auto& m : moves) {
+    int rc = order_after_block(s, s->blocks[m.bi], stream, &waited);
+    if (rc) { undo(); return rc; }
+  }
+  cudaError_t e = cudaSuccess;
+  if (moves.size() == 1) {
+    // parameters and optimizer state are one contiguous range; the step counter is host state
+    Block& b = s->blocks[moves[0].bi];
+    e = cudaMemcpyAsync(s->ctxs[dst_ctx].base + moves[0].noff, s->ctxs[b.ctx].base + b.off, b.bytes,
+                        cudaMemcpyDeviceToDevice, stream);
+  } else {
+    for (size_t first = 0; first < moves.size() && e == cudaSuccess; first += kMigPerLaunch) {
+      MigArgs a;
+      a.n = (int)std::min<size_t>(kMigPerLaunch, moves.size() - first);
+      unsigned int tiles = 0;
+      for (int k = 0; k < a.n; ++k) {
+        Block& b = s->blocks[moves[first + k].bi];
+        a.src[k] = reinterpret_cast<const unsigned char*>(s->ctxs[b.ctx].base + b.off);
+        a.dst[k] = reinterpret_cast<unsigned char*>(s->ctxs[dst_ctx].base + moves[first + k].noff);
+        a.bytes[k] = b.bytes;
+        a.tile_prefix[k] = tiles;
+        tiles += (unsigned int)((b.bytes + kMigTile - 1) / kMigTile);
+      }
+      a.tile_prefix[a.n] = tiles;
+      const int grid = (int)std::min<unsigned int>(tiles, (unsigned int)s->num_sms * 8u);
+      ps_migrate_kernel<<<grid, 256, 0, stream>>>(a);
+      e = cudaGetLastError();
+    }
+  }
+  if (e == cudaSuccess) e = cudaEventRecord(s->batches[batch].ev, stream);
+  if (e != cudaSuccess) { undo(); s->cuda_err = cudaGetErrorString(e); return PS_ERR_CUDA; }
+  MigBatch& mb = s->batches[batch];
+  mb.pending = true;
+  mb.seen_call = mb.waited_call = 0;
+  for (auto& m : moves) {
+    Block& b = s->blocks[m.bi];
+    s->pending_free.push_back(PendingFree{b.ctx, b.off, b.bytes, batch});
+    b.ctx = dst_ctx;
+    b.off = m.noff;
+    b.mig_batch = batch;
+  }
   return PS_OK;
 }
 
@@ -869,42 +986,28 @@ int ps_migrate_block(ps_service* s, int job, int block, int dst_ctx, void* strea
   const int bi = find_block(s, job, block);
   if (bi < 0 || dst_ctx < 0 || dst_ctx >= (int)s->ctxs.size()) return PS_ERR_BAD_ARG;
   if (!has_device(s)) return PS_ERR_NO_DEVICE;
-  Block& b = s->blocks[bi];
-  if (b.ctx == dst_ctx) return PS_OK;
   PS_CUDA(s, cudaSetDevice(s->device));
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  if (b.mig_pending) {   // a second move before the first copy landed: let it land
-    PS_CUDA(s, cudaEventSynchronize(b.mig_event));
-    b.mig_pending = false;
-    int rc0 = reap_frees(s, false);
-    if (rc0) return rc0;
+  ++s->call_id;
+  return migrate_many(s, std::vector<int>{bi}, dst_ctx, static_cast<cudaStream_t>(stream_));
+}
+
+int ps_migrate_blocks(ps_service* s, const ps_task* tasks, int n, int dst_ctx, void* stream_) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (n < 0 || (n > 0 && !tasks) || dst_ctx < 0 || dst_ctx >= (int)s->ctxs.size()) return PS_ERR_BAD_ARG;
+  std::vector<int> bis;
+  const unsigned long long gen = ++s->gen;
+  for (int i = 0; i < n; ++i) {
+    const int bi = find_block(s, tasks[i].job, tasks[i].block);
+    if (bi < 0) return PS_ERR_BAD_ARG;
+    if (s->blocks[bi].mark == gen) return PS_ERR_DUPLICATE;
+    s->blocks[bi].mark = gen;
+    bis.push_back(bi);
   }
-  size_t noff = 0;
-  int rc = arena_alloc(s, dst_ctx, b.bytes, &noff);
-  if (rc) return rc;
-  if (!b.mig_event) {
-    cudaError_t e = cudaEventCreateWithFlags(&b.mig_event, cudaEventDisableTiming);
-    if (e != cudaSuccess) {
-      s->ctxs[dst_ctx].arena.release(noff, b.bytes);
-      s->cuda_err = cudaGetErrorString(e);
-      return PS_ERR_CUDA;
-    }
-  }
-  rc = order_after_block(s, b, stream);
-  cudaError_t e = cudaSuccess;
-  if (!rc) {
-    // parameters, optimizer state (one contiguous range); the step counter is host state
-    e = cudaMemcpyAsync(s->ctxs[dst_ctx].base + noff, s->ctxs[b.ctx].base + b.off, b.bytes,
-                        cudaMemcpyDeviceToDevice, stream);
-    if (e == cudaSuccess) e = cudaEventRecord(b.mig_event, stream);
-    if (e != cudaSuccess) { s->cuda_err = cudaGetErrorString(e); rc = PS_ERR_CUDA; }
-  }
-  if (rc) { s->ctxs[dst_ctx].arena.release(noff, b.bytes); return rc; }
-  s->pending_free.push_back(PendingFree{b.ctx, b.off, b.bytes, b.mig_event, bi});
-  b.ctx = dst_ctx;
-  b.off = noff;
-  b.mig_pending = true;
-  return PS_OK;
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  PS_CUDA(s, cudaSetDevice(s->device));
+  ++s->call_id;
+  return migrate_many(s, bis, dst_ctx, static_cast<cudaStream_t>(stream_));
 }
 
 int ps_block_stats(ps_service* s, int job, int block, double* sq_out, unsigned long long* step_out) {

@@ -204,10 +204,14 @@ class SampledPair:
         torch.cuda.synchronize(self.dev)
 
     def migrate(self, plan, stream=None):
+        """Moves every listed block to the next context: one batched call per destination."""
+        by_dst = {}
         for (j, b) in plan:
             dst = (self.ctx[(j, b)] + 1) % self.cfg.num_contexts
-            self.svc.migrate_block(j, b, dst, stream)
+            by_dst.setdefault(dst, []).append((j, b))
             self.ctx[(j, b)] = dst
+        for dst, tasks in by_dst.items():
+            self.svc.migrate_blocks(tasks, dst, stream)
 
     def _gather(self, j: int):
         """p, s0, s1 of job j at the sampled positions, from the service's memory."""

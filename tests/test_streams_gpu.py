@@ -129,3 +129,53 @@ def test_concurrent_host_threads_are_serialised_by_the_service():
         pair.compare()
     finally:
         pair.close()
+
+
+def test_batched_migration_is_all_or_nothing_and_chains_without_host_waits():
+    sizes = [300_000, 5, 70_000, 1 << 20, 4096, 123_457] * 20          # 120 blocks: two gather launches per batch
+    cfg = tiny_config(sizes, 2)
+    cfg.num_contexts = 3
+    pair = Pair(cfg)
+    svc = pair.svc
+    try:
+        every = configs.rounds_all(cfg)[0]
+        pair.push_iteration(0)
+        pair.aggregate(every)
+        with pytest.raises(B.PsError) as e:
+            svc.migrate_blocks(every + [every[0]], 1)
+        assert e.value.status == B.PS_ERR_DUPLICATE
+        with pytest.raises(B.PsError) as e:
+            svc.migrate_blocks(every, 7)
+        assert e.value.status == B.PS_ERR_BAD_ARG
+        side = torch.cuda.Stream()
+        # everything to context 2, then straight on to context 0 and back to 1: each batch is ordered
+        # after the previous one on the device, the host never waits
+        for dst in (2, 0, 1):
+            svc.migrate_blocks(every, dst, side)
+            for (j, b) in every:
+                pair.ora.migrate_block(j, b, dst)
+        pair.push_iteration(1)
+        pair.aggregate(every)                           # default stream: must wait for the last batch
+        pair.compare()
+        assert all(svc.block_state(0, b)[2] == 1 for _, b in every)
+        torch.cuda.synchronize()
+        used = [svc.arena_info(c)[0] for c in range(3)]
+        assert used[0] == 0 and used[2] == 0 and used[1] > 0          # the sources were released
+        # a destination without room for the whole batch: nothing moves
+        tiny = B.Service(0, 2, (1 << 20) + (1 << 19))
+        try:
+            j = tiny.register_job(num_workers=1)
+            for b in range(3):
+                tiny.register_block(j, b, 60_000, 0)                  # 3 x 480,256 bytes in context 0
+            tiny.register_block(j, 3, 60_000, 1)                      # context 1 has room for two more only
+            with pytest.raises(B.PsError) as e:
+                tiny.migrate_blocks([(j, 0), (j, 1), (j, 2)], 1)
+            assert e.value.status == B.PS_ERR_NOMEM
+            assert [tiny.block_state(j, b)[2] for b in range(4)] == [0, 0, 0, 1]
+            assert tiny.arena_info(1)[0] == 480_256
+            tiny.migrate_blocks([(j, 0), (j, 2)], 1)
+            assert [tiny.block_state(j, b)[2] for b in range(4)] == [1, 0, 1, 1]
+        finally:
+            tiny.close()
+    finally:
+        pair.close()
