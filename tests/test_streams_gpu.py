@@ -76,15 +76,16 @@ def test_maximum_worker_count(dt):
         pair.close()
 
 
-def test_destroy_with_work_in_flight_and_handle_reuse_is_rejected():
+def test_destroy_with_work_in_flight():
     cfg = tiny_config([1 << 21], 8)
     pair = Pair(cfg)
     pair.push_iteration(0)
     pair.svc.aggregate([(0, 0)], torch.cuda.Stream())
-    handle = pair.svc.handle
-    pair.close()                                        # waits for the launch, then frees
-    torch.cuda.synchronize()
-    assert handle is not None
+    pair.close()                                        # waits for the launch, then frees everything
+    torch.cuda.synchronize()                            # the context is still healthy
+    x = torch.ones(16, device="cuda")
+    assert float(x.sum()) == 16.0
+    assert B.load().ps_destroy(None) == B.PS_ERR_BAD_HANDLE
 
 
 def test_one_very_large_block():
