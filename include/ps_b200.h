@@ -347,6 +347,9 @@ int ps_planner_assign(ps_planner* pl, int job, double exec_time, int* task_out, 
  * Aggregator through ps_planner_task_info (the caller migrates the blocks). */
 int ps_planner_remove_job(ps_planner* pl, int job, int* released_out);
 int ps_planner_task_info(ps_planner* pl, int task, int* job_out, int* aggregator_out, double* exec_time_out);
+/* Cyclic execution (Section 3.3.1): how many times the task runs in one cycle of
+ * its Aggregator, floor(C_n / d_j), and the period d_j of its slots there. */
+int ps_planner_task_runs(ps_planner* pl, int task, int* runs_per_cycle_out, double* slot_period_out);
 /* cycle = C_n; load = W_n = sum_j floor(C_n/d_j) * sum e_t (Appendix C). */
 int ps_planner_aggregator_info(ps_planner* pl, int aggregator, int* alive_out, double* cycle_out,
                                double* load_out, int* num_tasks_out);

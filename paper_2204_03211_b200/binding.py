@@ -90,6 +90,7 @@ _SIGNATURES = {
     "ps_planner_remove_job": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int)]),
     "ps_planner_task_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int),
                                        C.POINTER(C.c_double)]),
+    "ps_planner_task_runs": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_double)]),
     "ps_planner_aggregator_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_double),
                                              C.POINTER(C.c_double), C.POINTER(C.c_int)]),
     "ps_planner_job_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double),
@@ -363,6 +364,11 @@ class Planner:
         _check(load().ps_planner_task_info(self.handle, task, C.byref(j), C.byref(n), C.byref(e)),
                "ps_planner_task_info")
         return j.value, n.value, e.value
+
+    def task_runs(self, task: int):
+        r, d = C.c_int(), C.c_double()
+        _check(load().ps_planner_task_runs(self.handle, task, C.byref(r), C.byref(d)), "ps_planner_task_runs")
+        return r.value, d.value
 
     def aggregator_info(self, n: int):
         a, c, w, k = C.c_int(), C.c_double(), C.c_double(), C.c_int()

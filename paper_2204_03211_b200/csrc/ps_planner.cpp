@@ -243,6 +243,18 @@ int ps_planner_task_info(ps_planner* p, int task, int* job_out, int* aggregator_
   return PS_OK;
 }
 
+int ps_planner_task_runs(ps_planner* p, int task, int* runs_per_cycle_out, double* slot_period_out) {
+  if (!ok(p)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(p->mu);
+  if (task < 0 || task >= (int)p->tasks.size() || !p->tasks[task].alive) return PS_ERR_BAD_ARG;
+  const Task& t = p->tasks[task];
+  const double C = p->cycle(t.agg);
+  const double d = stretched(p->D[t.job], C);
+  if (runs_per_cycle_out) *runs_per_cycle_out = (int)floor_div(C, d);
+  if (slot_period_out) *slot_period_out = d;
+  return PS_OK;
+}
+
 int ps_planner_aggregator_info(ps_planner* p, int aggregator, int* alive_out, double* cycle_out, double* load_out,
                                int* num_tasks_out) {
   if (!ok(p)) return PS_ERR_BAD_HANDLE;

@@ -168,6 +168,8 @@ def test_planner_reproduces_the_papers_toy_numbers(_lib):
     info = p.aggregator_info(n1)
     assert n2 == n1 and info["cycle"] == g["A.cycle_packed"] and info["load"] == 2 * g["A.e1"] + g["A.e2"]
     assert p.job_info(j1)["loss"] == 0.0 and p.num_aggregators() == (1, 1)
+    assert p.task_runs(0) == (int(g["A.runs_of_J1_per_cycle"]), g["A.D1"])      # J1's task: twice per cycle of 12
+    assert p.task_runs(1) == (1, g["A.D2"])
     q = B.Planner(g["loss_limit"])
     a, b = q.add_job(g["B.D"]), q.add_job(g["A.D2"])
     _, n0 = q.assign(a, g["B.e"])
