@@ -76,6 +76,20 @@ __device__ __forceinline__ void update4(const Hp& h, const float4& G, float* p, 
 
 // ---------------------------------------------------------------- chunk bodies
 // NT = number of cooperating threads, tid = this thread's index among them.
+//
+// The vector bodies are bound by memory latency, not by issue slots: a thread
+// cannot hold enough 128-bit loads in registers to cover the HBM latency at
+// full occupancy.  So lines are requested ahead of their use with L2
+// prefetches, which occupy no register: the demand loads then complete from
+// L2.  One lane per 128-byte line issues the prefetch; every prefetched
+// address is one that a demand load of the same chunk reads later.
+
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+constexpr int kAheadF32 = 2;         // fp32 shards: workers requested ahead inside the worker loop
+constexpr int kAheadBf16 = 4;        // bf16 shards: the same
+constexpr int kNextTripMaxW = 8;     // up to this many workers the loop is too short to run ahead in: the
+                                     // next trip's first lines are requested at the top of each trip instead
 
 // fp32 gradients, 16-byte aligned: each thread owns U float4 groups per trip.
 template <int OPT, int U, int NT>
@@ -83,6 +97,7 @@ __device__ __forceinline__ void chunk_f32_vec(unsigned int tid, const Hp& h, con
                                               int W, float* __restrict__ p, float* __restrict__ s0,
                                               float* __restrict__ s1, size_t begin, unsigned int count, double& sq) {
   const unsigned int nvec = count >> 2;
+  const bool pf_lane = (tid & 7) == 0;      // 8 lanes x 16 bytes = one line
   unsigned int i = tid;
   // full trips: U groups per thread, no predicates
   for (; i + (U - 1) * NT < nvec; i += U * NT) {
@@ -94,13 +109,43 @@ __device__ __forceinline__ void chunk_f32_vec(unsigned int tid, const Hp& h, con
       av[u] = *reinterpret_cast<const float4*>(s0 + e);
       if (OPT == 1) bv[u] = *reinterpret_cast<const float4*>(s1 + e); else bv[u] = make_float4(0, 0, 0, 0);
     }
+    if (pf_lane) {
+      if (W <= kNextTripMaxW && i + U * NT + (U - 1) * NT < nvec) {
+        // next full trip: parameters, state and the first shards
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const size_t e = begin + 4 * (size_t)(i + (U + u) * NT);
+          prefetch_l2(p + e);
+          prefetch_l2(s0 + e);
+          if (OPT == 1) prefetch_l2(s1 + e);
+        }
+        for (int w = 0; w <= kAheadF32 && w < W; ++w) {
+          const float* g = static_cast<const float*>(ld_ptr(shards, w));
+#pragma unroll
+          for (int u = 0; u < U; ++u) prefetch_l2(g + begin + 4 * (size_t)(i + (U + u) * NT));
+        }
+      }
+      if (W > kNextTripMaxW || i == tid) {
+        // this trip's first shards after shard 0 (not requested by an earlier trip)
+        for (int w = 1; w <= kAheadF32 && w < W; ++w) {
+          const float* g = static_cast<const float*>(ld_ptr(shards, w));
+#pragma unroll
+          for (int u = 0; u < U; ++u) prefetch_l2(g + begin + 4 * (size_t)(i + u * NT));
+        }
+      }
+    }
     {
       const float* g = static_cast<const float*>(ld_ptr(shards));
 #pragma unroll
       for (int u = 0; u < U; ++u) acc[u] = as_f4(ld_stream(g + begin + 4 * (size_t)(i + u * NT)));
     }
-#pragma unroll 4
+#pragma unroll 2
     for (int w = 1; w < W; ++w) {
+      if (pf_lane && w + kAheadF32 < W) {
+        const float* ga = static_cast<const float*>(ld_ptr(shards, w + kAheadF32));
+#pragma unroll
+        for (int u = 0; u < U; ++u) prefetch_l2(ga + begin + 4 * (size_t)(i + u * NT));
+      }
       const float* g = static_cast<const float*>(ld_ptr(shards, w));
 #pragma unroll
       for (int u = 0; u < U; ++u) acc[u] = add4(acc[u], ld_stream(g + begin + 4 * (size_t)(i + u * NT)));
@@ -123,28 +168,41 @@ __device__ __forceinline__ void chunk_f32_vec(unsigned int tid, const Hp& h, con
 }
 
 // bf16 gradients, 16-byte aligned: each thread owns 8 consecutive elements.
+// Parameters and state are requested at the top of a trip and loaded after the
+// worker loop, so their 24 registers are free while the shards stream.
 template <int OPT, int NT>
 __device__ __forceinline__ void chunk_bf16_vec(unsigned int tid, const Hp& h, const void* const* __restrict__ shards,
                                                int W, float* __restrict__ p, float* __restrict__ s0,
                                                float* __restrict__ s1, size_t begin, unsigned int count, double& sq) {
   const unsigned int nvec = count >> 3;
+  const bool pf_lane = (tid & 7) == 0;      // shards: 8 lanes x 16 bytes = one line
   for (unsigned int i = tid; i < nvec; i += NT) {
     const size_t e = begin + 8 * (size_t)i;
+    if ((tid & 3) == 0) {                   // parameters and state: 4 lanes x 32 bytes = one line
+      prefetch_l2(p + e);
+      prefetch_l2(s0 + e);
+      if (OPT == 1) prefetch_l2(s1 + e);
+    }
+    if (pf_lane)
+      for (int w = 1; w <= kAheadBf16 && w < W; ++w)
+        prefetch_l2(static_cast<const unsigned short*>(ld_ptr(shards, w)) + e);
+    float acc[8];
+    widen8(ld_stream(static_cast<const unsigned short*>(ld_ptr(shards)) + e), acc);
+#pragma unroll 2
+    for (int w = 1; w < W; ++w) {
+      if (pf_lane && w + kAheadBf16 < W)
+        prefetch_l2(static_cast<const unsigned short*>(ld_ptr(shards, w + kAheadBf16)) + e);
+      float g[8];
+      widen8(ld_stream(static_cast<const unsigned short*>(ld_ptr(shards, w)) + e), g);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
+    }
     const float4 p0 = *reinterpret_cast<const float4*>(p + e), p1 = *reinterpret_cast<const float4*>(p + e + 4);
     const float4 a0 = *reinterpret_cast<const float4*>(s0 + e), a1 = *reinterpret_cast<const float4*>(s0 + e + 4);
     float4 b0 = make_float4(0, 0, 0, 0), b1 = b0;
     if (OPT == 1) {
       b0 = *reinterpret_cast<const float4*>(s1 + e);
       b1 = *reinterpret_cast<const float4*>(s1 + e + 4);
-    }
-    float acc[8];
-    widen8(ld_stream(static_cast<const unsigned short*>(ld_ptr(shards)) + e), acc);
-#pragma unroll 2   // measured on B200 (W = 32): 2 beats 4, 8 and 16
-    for (int w = 1; w < W; ++w) {
-      float g[8];
-      widen8(ld_stream(static_cast<const unsigned short*>(ld_ptr(shards, w)) + e), g);
-#pragma unroll
-      for (int k = 0; k < 8; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
     }
     update4<OPT>(h, make_float4(acc[0], acc[1], acc[2], acc[3]), p, s0, s1, e, p0, a0, b0, sq);
     update4<OPT>(h, make_float4(acc[4], acc[5], acc[6], acc[7]), p, s0, s1, e + 4, p1, a1, b1, sq);
