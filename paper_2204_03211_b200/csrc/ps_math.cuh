@@ -34,6 +34,21 @@ __device__ __forceinline__ void update_elem(const Hp& h, float G, float& p, floa
 __device__ __forceinline__ float bf16_lo(unsigned int u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(unsigned int u) { return __uint_as_float(u & 0xffff0000u); }
 
+// lo += bf16(low half of u), hi += bf16(high half of u).  The mixed-precision
+// add widens its bf16 operand exactly and rounds the binary32 sum once to
+// nearest-even (subnormals kept), i.e. the same bits as
+// __fadd_rn(acc, bf16_lo/hi(u)) with one instruction per element instead of two.
+__device__ __forceinline__ void add_bf16x2(float& lo, float& hi, unsigned int u) {
+  asm("{\n\t"
+      ".reg .b16 l, h;\n\t"
+      "mov.b32 {l, h}, %2;\n\t"
+      "add.rn.f32.bf16 %0, l, %0;\n\t"
+      "add.rn.f32.bf16 %1, h, %1;\n\t"
+      "}"
+      : "+f"(lo), "+f"(hi)
+      : "r"(u));
+}
+
 // Shard pointer w of a task (uniform across the CTA).  A generic load: the
 // pointer row may sit in the global task table or in shared memory.
 __device__ __forceinline__ const void* ld_ptr(const void* const* shards, int w = 0) {
@@ -188,14 +203,15 @@ __device__ __forceinline__ void chunk_bf16_vec(unsigned int tid, const Hp& h, co
         prefetch_l2(static_cast<const unsigned short*>(ld_ptr(shards, w)) + e);
     float acc[8];
     widen8(ld_stream(static_cast<const unsigned short*>(ld_ptr(shards)) + e), acc);
-#pragma unroll 2
+#pragma unroll 4
     for (int w = 1; w < W; ++w) {
       if (pf_lane && w + kAheadBf16 < W)
         prefetch_l2(static_cast<const unsigned short*>(ld_ptr(shards, w + kAheadBf16)) + e);
-      float g[8];
-      widen8(ld_stream(static_cast<const unsigned short*>(ld_ptr(shards, w)) + e), g);
-#pragma unroll
-      for (int k = 0; k < 8; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
+      const uint4 t = ld_stream(static_cast<const unsigned short*>(ld_ptr(shards, w)) + e);
+      add_bf16x2(acc[0], acc[1], t.x);
+      add_bf16x2(acc[2], acc[3], t.y);
+      add_bf16x2(acc[4], acc[5], t.z);
+      add_bf16x2(acc[6], acc[7], t.w);
     }
     const float4 p0 = *reinterpret_cast<const float4*>(p + e), p1 = *reinterpret_cast<const float4*>(p + e + 4);
     const float4 a0 = *reinterpret_cast<const float4*>(s0 + e), a1 = *reinterpret_cast<const float4*>(s0 + e + 4);

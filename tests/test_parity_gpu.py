@@ -91,6 +91,43 @@ def test_c1_ten_iterations(kernel):
         pair.close()
 
 
+@pytest.mark.parametrize("opt", [configs.SGD, configs.ADAM])
+def test_bf16_every_bit_pattern_sums_like_the_oracle(opt):
+    """The vector path adds bf16 shards with a widening add instruction; the
+    oracle widens (bits << 16) and adds in binary32.  Every one of the 65,536
+    bf16 patterns meets finite, subnormal, huge and infinite partners here."""
+    reps, W = 4, 3
+    n = 65536 * reps
+    cfg = tiny_config([n], W, opt=opt, grad_dtype=configs.BF16, weight_decay=0.0)
+    pair = Pair(cfg)
+    try:
+        rng = np.random.default_rng(77)
+        every = np.tile(np.arange(65536, dtype=np.uint16), reps)
+        partner = rng.integers(0, 65536, n, dtype=np.uint16)
+        partner[:65536] &= 0x807F                      # subnormal or zero partners for the first copy
+        partner[65536:2 * 65536] = (partner[65536:2 * 65536] & 0x80FF) | 0x3A00   # around 1e-3
+        third = rng.integers(0, 65536, n, dtype=np.uint16)
+        third[2 * 65536:3 * 65536] = 0x0001            # the smallest subnormal
+        shards = [partner, every, third]
+        dev = []
+        for w, a in enumerate(shards):
+            t = torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16).cuda()
+            dev.append(t)
+            pair.svc.push(0, 0, w, t)
+            pair.ora.push(0, 0, w, a)
+        pair.aggregate([(0, 0)])
+        p, a, v, _ = pair.gpu_block(0, 0)
+        rp = pair.ora.pull(0, 0)
+        ra, rv = pair.ora.state(0, 0)
+        for got, ref in ((p, rp), (a, ra)) + (((v, rv),) if rv is not None else ()):
+            nan = np.isnan(ref)
+            assert np.array_equal(np.isnan(got), nan)
+            assert np.array_equal(got[~nan].view(np.uint32), ref[~nan].view(np.uint32))
+        assert (~np.isnan(ra)).sum() > n // 2
+    finally:
+        pair.close()
+
+
 def test_results_repeat_bit_for_bit_across_runs():
     outs = []
     for _ in range(2):
