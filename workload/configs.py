@@ -176,6 +176,8 @@ def rounds_poisson(cfg: Config, iteration: int, ticks: int = 16) -> list:
 
 
 def rounds_for(cfg: Config, iteration: int, ticks: int = 16) -> list:
+    if ticks == 1:          # one round: everything is ready at once, whatever the arrival pattern
+        return rounds_all(cfg)
     if cfg.arrival == "reverse_layer":
         return rounds_reverse_layer(cfg)
     if cfg.arrival == "poisson":
