@@ -88,6 +88,9 @@ enum {
                               ps_block_stats, ps_block_profile, ps_migrate_block and ps_push_host
                               order themselves after the block's last launch in either mode.
                               Default 0: every launch is enqueued on `stream` itself. */
+  PS_OPT_INLINE_TABLE = 7, /* 1 (default): a launch whose task table fits 3968 bytes (a round of a few
+                              tensors) and has few chunks passes the table as a kernel parameter, one
+                              CTA per chunk: no upload.  0: always upload the table.  Same results. */
   PS_OPT_PROFILE = 5,      /* 1: aggregates record per-task device time (see ps_block_profile);
                               costs a few atomics per chunk; direct-load kernel only; default 0 */
   PS_OPT_KERNEL = 4        /* kernel variant: 0 = automatic (direct loads), 1 = direct loads,

@@ -25,6 +25,7 @@ PS_DEVICE_NONE = -1
 PS_MAX_WORKERS = 256
 PS_OPT_CHUNK_ELEMS, PS_OPT_CTAS_PER_SM, PS_OPT_SORT_TASKS, PS_OPT_KERNEL, PS_OPT_PROFILE = 1, 2, 3, 4, 5
 PS_OPT_OVERLAP = 6
+PS_OPT_INLINE_TABLE = 7
 
 
 class ps_job_desc(C.Structure):

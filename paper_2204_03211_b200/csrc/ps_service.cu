@@ -27,7 +27,15 @@
 namespace psb {
 
 constexpr uint32_t kMagic = 0x50534232u;   // "PSB2"
-constexpr int kSlots = 4;                  // task tables in flight
+#ifndef PS_SLOTS
+#define PS_SLOTS 8
+#endif
+#ifndef PS_WORK_STREAMS
+#define PS_WORK_STREAMS 4
+#endif
+constexpr int kSlots = PS_SLOTS;           // task tables in flight
+constexpr int kInlineGridFactor = 4;         // an inline launch has at most this many CTAs per resident slot
+constexpr int kWorkStreams = PS_WORK_STREAMS;   // overlap mode: launches rotate over this many streams
 constexpr unsigned int kMaxChunk = 1u << 20;
 
 struct Job {
@@ -88,6 +96,7 @@ struct Slot {
   size_t cap = 0;
   double* partials = nullptr;
   size_t partial_cap = 0;
+  PsTaskMut* mut = nullptr;                // per-task state of launches whose table travels as a kernel parameter
   cudaEvent_t done = nullptr;
   cudaEvent_t copied = nullptr;            // table upload finished (recorded on the copy stream)
   cudaEvent_t input = nullptr;             // overlap mode: the caller's stream at the time of the call
@@ -127,10 +136,11 @@ struct ps_service {
   long long opt_chunk = 0, opt_ctas = 0, opt_sort = 1, opt_kernel = 0, opt_profile = 0;
   int* status_dev = nullptr;               // error word written by kernels whose waits expired
   cudaStream_t copy_stream = nullptr;      // table uploads run here, beside the previous launch
-  cudaStream_t work_streams[2] = {nullptr, nullptr};   // overlap mode: launches alternate between these
+  cudaStream_t work_streams[kWorkStreams] = {};   // overlap mode: launches rotate over these
   int next_work = 0;
   unsigned int unjoined = 0;               // overlap mode: slots whose launch no caller stream has joined yet
   long long opt_overlap = 0;
+  long long opt_inline = 1;               // small launches carry their table as a kernel parameter
   int occ_ctas = 0;
   unsigned long long launches = 0;
   int last_grid = 0, last_block = 0;
@@ -439,6 +449,10 @@ int acquire_slot(ps_service* s, size_t table_bytes, size_t nchunks, Slot** out) 
     PS_CUDA(s, cudaMalloc(&sl.partials, ncap * sizeof(double)));
     sl.partial_cap = ncap;
   }
+  if (!sl.mut) {
+    PS_CUDA(s, cudaMalloc(&sl.mut, kInlineMaxTasks * sizeof(PsTaskMut)));
+    PS_CUDA(s, cudaMemset(sl.mut, 0, kInlineMaxTasks * sizeof(PsTaskMut)));   // kept all-zero by the kernel
+  }
   sl.gen = s->gen;
   *out = &sl;
   return PS_OK;
@@ -506,7 +520,7 @@ int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(ps_aggregate_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBulkSmemBytes);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking);
-    for (int i = 0; i < 2 && e == cudaSuccess; ++i)
+    for (int i = 0; i < kWorkStreams && e == cudaSuccess; ++i)
       e = cudaStreamCreateWithFlags(&s->work_streams[i], cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaMalloc(&s->status_dev, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(s->status_dev, 0, sizeof(int));
@@ -543,6 +557,7 @@ int ps_destroy(ps_service* s) {
       if (sl.host) cudaFreeHost(sl.host);
       if (sl.dev) cudaFree(sl.dev);
       if (sl.partials) cudaFree(sl.partials);
+      if (sl.mut) cudaFree(sl.mut);
       if (sl.done) cudaEventDestroy(sl.done);
       if (sl.copied) cudaEventDestroy(sl.copied);
       if (sl.input) cudaEventDestroy(sl.input);
@@ -764,16 +779,21 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
   if (rc) return rc;
   Slot* sl = nullptr;
   const bool bulk = use_bulk(s) && !plan.has_sparse;
-  rc = acquire_slot(s, plan.bytes.size(), (size_t)plan.total_chunks * (bulk ? kBulkConsumerWarps : 1), &sl);
+  // A small table (a round of a few tensors) travels as a kernel parameter: no
+  // upload, no copy event, and one CTA per chunk instead of a work counter.
+  const bool inl = s->opt_inline && !bulk && !plan.has_sparse && plan.bytes.size() <= kInlineBytes &&
+                   plan.total_chunks <= (unsigned int)(kInlineGridFactor * grid_cap(s));
+  rc = acquire_slot(s, inl ? 0 : plan.bytes.size(),
+                    (size_t)plan.total_chunks * (bulk ? kBulkConsumerWarps : 1), &sl);
   if (rc) return rc;
   const int slot_index = (int)(sl - s->slots);
-  // Overlap mode: the launch goes to one of two service-owned streams, after the
+  // Overlap mode: the launch goes to one of the service-owned streams, after the
   // work the caller has enqueued on `stream` so far; consecutive launches then
   // overlap (the next one's CTAs fill the SMs the previous one's tail leaves idle).
   cudaStream_t run = stream;
   if (s->opt_overlap) {
     run = s->work_streams[s->next_work];
-    s->next_work ^= 1;
+    s->next_work = (s->next_work + 1) % kWorkStreams;
     PS_CUDA(s, cudaEventRecord(sl->input, stream));
     PS_CUDA(s, cudaStreamWaitEvent(run, sl->input, 0));
   }
@@ -782,18 +802,25 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
     rc = order_after_block(s, s->blocks[bi], run, &waited);
     if (rc) return rc;
   }
-  std::memcpy(sl->host, plan.bytes.data(), plan.bytes.size());
-  // The table depends on nothing the caller enqueued, so its upload goes to the
-  // service's own stream and overlaps the previous launch; the kernel waits for it.
-  PS_CUDA(s, cudaMemcpyAsync(sl->dev, sl->host, plan.bytes.size(), cudaMemcpyHostToDevice, s->copy_stream));
-  PS_CUDA(s, cudaEventRecord(sl->copied, s->copy_stream));
-  PS_CUDA(s, cudaStreamWaitEvent(run, sl->copied, 0));
-  const int grid = (int)std::min<unsigned long long>(plan.total_chunks, (unsigned long long)grid_cap(s));
-  if (bulk)
-    ps_aggregate_bulk_kernel<<<grid, kBulkThreads, kBulkSmemBytes, run>>>(sl->dev, s->jobs_dev, s->stats_dev,
-                                                                          sl->partials, s->status_dev);
-  else
-    ps_aggregate_ldg_kernel<<<grid, kThreads, 0, run>>>(sl->dev, s->jobs_dev, s->stats_dev, sl->partials);
+  int grid = (int)std::min<unsigned long long>(plan.total_chunks, (unsigned long long)grid_cap(s));
+  if (inl) {
+    PsInlineTable tbl;
+    std::memcpy(tbl.bytes, plan.bytes.data(), plan.bytes.size());
+    grid = (int)plan.total_chunks;
+    ps_aggregate_inline_kernel<<<grid, kThreads, 0, run>>>(tbl, s->jobs_dev, s->stats_dev, sl->partials, sl->mut);
+  } else {
+    std::memcpy(sl->host, plan.bytes.data(), plan.bytes.size());
+    // The table depends on nothing the caller enqueued, so its upload goes to the
+    // service's own stream and overlaps the previous launch; the kernel waits for it.
+    PS_CUDA(s, cudaMemcpyAsync(sl->dev, sl->host, plan.bytes.size(), cudaMemcpyHostToDevice, s->copy_stream));
+    PS_CUDA(s, cudaEventRecord(sl->copied, s->copy_stream));
+    PS_CUDA(s, cudaStreamWaitEvent(run, sl->copied, 0));
+    if (bulk)
+      ps_aggregate_bulk_kernel<<<grid, kBulkThreads, kBulkSmemBytes, run>>>(sl->dev, s->jobs_dev, s->stats_dev,
+                                                                            sl->partials, s->status_dev);
+    else
+      ps_aggregate_ldg_kernel<<<grid, kThreads, 0, run>>>(sl->dev, s->jobs_dev, s->stats_dev, sl->partials);
+  }
   PS_CUDA(s, cudaGetLastError());
   PS_CUDA(s, cudaEventRecord(sl->done, run));
   sl->inflight = true;
@@ -802,7 +829,7 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
   s->launches++;
   s->last_grid = grid;
   s->last_block = bulk ? kBulkThreads : kThreads;
-  s->last_kernel = bulk ? "bulk" : "ldg";
+  s->last_kernel = inl ? "inline" : bulk ? "bulk" : "ldg";
   for (int bi : idx) {
     Block& b = s->blocks[bi];
     b.step++;
@@ -1114,6 +1141,9 @@ int ps_set_option(ps_service* s, int option, long long value) {
     case PS_OPT_OVERLAP:
       s->opt_overlap = value ? 1 : 0;
       return PS_OK;
+    case PS_OPT_INLINE_TABLE:
+      s->opt_inline = value ? 1 : 0;
+      return PS_OK;
     default:
       return PS_ERR_BAD_ARG;
   }
@@ -1130,6 +1160,7 @@ int ps_get_option(ps_service* s, int option, long long* out) {
     case PS_OPT_KERNEL: *out = s->opt_kernel; return PS_OK;
     case PS_OPT_PROFILE: *out = s->opt_profile; return PS_OK;
     case PS_OPT_OVERLAP: *out = s->opt_overlap; return PS_OK;
+    case PS_OPT_INLINE_TABLE: *out = s->opt_inline; return PS_OK;
     default: return PS_ERR_BAD_ARG;
   }
 }

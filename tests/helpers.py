@@ -41,7 +41,11 @@ class Pair:
         self.dev = torch.device("cuda", device)
         need = sum(3 * (4 * b.nelem + 256) for j in cfg.jobs for b in j.blocks) + (1 << 20)
         self.svc = B.Service(device, cfg.num_contexts, arena_bytes or need)
-        self.svc.set_option(B.PS_OPT_KERNEL, kernel)
+        # kernel: 0 automatic, 1 direct loads with an uploaded table, 2 bulk-copy ring,
+        # 3 direct loads with the table passed as a kernel parameter where it fits
+        self.svc.set_option(B.PS_OPT_KERNEL, 1 if kernel == 3 else kernel)
+        if kernel in (1, 3):
+            self.svc.set_option(B.PS_OPT_INLINE_TABLE, int(kernel == 3))
         self.ora = A.OracleAggregator(cfg.num_contexts, nthreads)
         self.keep = []          # gradient tensors of the iteration in flight
         for j, job in enumerate(cfg.jobs):

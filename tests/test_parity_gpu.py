@@ -15,7 +15,7 @@ ODD_SIZES = [1, 3, 4, 5, 127, 1024, 4097, 12289, 70001]
 @pytest.mark.parametrize("opt,dt", [(configs.SGD, configs.F32), (configs.ADAM, configs.F32),
                                     (configs.SGD, configs.BF16), (configs.ADAM, configs.BF16)])
 @pytest.mark.parametrize("W", [1, 2, 5, 8, 33, 70])
-@pytest.mark.parametrize("kernel", [1, 2], ids=["ldg", "bulk"])
+@pytest.mark.parametrize("kernel", [1, 2, 3], ids=["ldg", "bulk", "inline"])
 def test_odd_sizes_bit_exact(opt, dt, W, kernel):
     # W = 70 with fp32 gradients exceeds what one ring stage can hold, so the
     # bulk-copy kernel hands those chunks to its direct-load path.
@@ -32,7 +32,7 @@ def test_odd_sizes_bit_exact(opt, dt, W, kernel):
 
 
 @pytest.mark.parametrize("chunk", [1024, 2048, 8192, 65536])
-@pytest.mark.parametrize("kernel", [1, 2], ids=["ldg", "bulk"])
+@pytest.mark.parametrize("kernel", [1, 2, 3], ids=["ldg", "bulk", "inline"])
 def test_chunk_size_and_order_invariance(chunk, kernel):
     cfg = tiny_config([5, 40000, 1024, 300001, 77], 4)
     pair = Pair(cfg, kernel=kernel)
@@ -48,7 +48,7 @@ def test_chunk_size_and_order_invariance(chunk, kernel):
         pair.close()
 
 
-@pytest.mark.parametrize("kernel", [1, 2], ids=["ldg", "bulk"])
+@pytest.mark.parametrize("kernel", [1, 2, 3], ids=["ldg", "bulk", "inline"])
 def test_unaligned_shards_take_scalar_path_same_bits(kernel):
     cfg = tiny_config([4099, 600], 3)
     pair = Pair(cfg, kernel=kernel)
@@ -76,7 +76,7 @@ def test_unaligned_shards_take_scalar_path_same_bits(kernel):
         pair.close()
 
 
-@pytest.mark.parametrize("kernel", [1, 2], ids=["ldg", "bulk"])
+@pytest.mark.parametrize("kernel", [1, 2, 3], ids=["ldg", "bulk", "inline"])
 def test_c1_ten_iterations(kernel):
     cfg = configs.c1()
     pair = Pair(cfg, kernel=kernel)
@@ -124,6 +124,41 @@ def test_bf16_every_bit_pattern_sums_like_the_oracle(opt):
             assert np.array_equal(np.isnan(got), nan)
             assert np.array_equal(got[~nan].view(np.uint32), ref[~nan].view(np.uint32))
         assert (~np.isnan(ra)).sum() > n // 2
+    finally:
+        pair.close()
+
+
+def test_small_rounds_travel_as_kernel_parameters_and_slots_stay_clean():
+    """A round whose table fits the kernel-parameter limit launches without an
+    upload.  Tasks of several chunks count their chunks in per-slot device
+    state that the finalizing CTA clears: twenty rounds reuse every slot, and
+    the per-block norm (summed by the finalizer) must be right every time."""
+    cfg = tiny_config([40000, 5, 70001, 1024], 4, opt=configs.ADAM)
+    pair = Pair(cfg, kernel=3)
+    try:
+        pair.svc.set_option(B.PS_OPT_PROFILE, 1)
+        every = configs.rounds_all(cfg)[0]
+        for it in range(20):
+            pair.push_iteration(it % 3)
+            if it == 0:
+                assert len(pair.svc.plan(every)) > 8      # several chunks per task
+            pair.aggregate(every if it % 2 else every[::-1])
+            assert pair.svc.launch_info()["kernel"] == "inline"
+            if it % 5 == 4 or it < 2:
+                pair.compare()
+                for b in range(4):
+                    busy, span = pair.svc.block_profile(0, b)
+                    assert 0.0 < busy < 1e5 and 0.0 < span < 1e5
+        # a table too large for the parameter space is uploaded as before
+        big = tiny_config([300] * 40, 4)
+        other = Pair(big, kernel=3)
+        try:
+            other.push_iteration(0)
+            other.aggregate(configs.rounds_all(big)[0])
+            assert other.svc.launch_info()["kernel"] == "ldg"
+            other.compare()
+        finally:
+            other.close()
     finally:
         pair.close()
 
