@@ -27,15 +27,9 @@
 namespace psb {
 
 constexpr uint32_t kMagic = 0x50534232u;   // "PSB2"
-#ifndef PS_SLOTS
-#define PS_SLOTS 8
-#endif
-#ifndef PS_WORK_STREAMS
-#define PS_WORK_STREAMS 4
-#endif
-constexpr int kSlots = PS_SLOTS;           // task tables in flight
+constexpr int kSlots = 8;                  // task tables in flight
 constexpr int kInlineGridFactor = 4;         // an inline launch has at most this many CTAs per resident slot
-constexpr int kWorkStreams = PS_WORK_STREAMS;   // overlap mode: launches rotate over this many streams
+constexpr int kWorkStreams = 4;             // overlap mode: launches rotate over this many streams
 constexpr unsigned int kMaxChunk = 1u << 20;
 
 struct Job {
@@ -987,7 +981,7 @@ static int migrate_many(ps_service* s, const std::vector<int>& bis, int dst_ctx,
         tiles += (unsigned int)((b.bytes + kMigTile - 1) / kMigTile);
       }
       a.tile_prefix[a.n] = tiles;
-      const int grid = (int)std::min<unsigned int>(tiles, (unsigned int)s->num_sms * 8u);
+      const int grid = (int)std::min<unsigned int>(tiles, (unsigned int)s->num_sms * 16u);
       ps_migrate_kernel<<<grid, 256, 0, stream>>>(a);
       e = cudaGetLastError();
     }
