@@ -3,7 +3,7 @@
 // the table's atomic counter, cuts each chunk into tiles and streams every
 // tile's rows — the W gradient shards, the parameters and the optimizer state —
 // into a shared-memory ring with 1-D bulk asynchronous copies (TMA unit,
-// completion counted on an mbarrier; no cluster multicast).  Eight consumer
+// completion counted on an mbarrier; every CTA fetches its own tiles).  Eight consumer
 // warps take tiles out of the ring, sum the shards in worker order 0..W-1 in
 // binary32, apply the optimizer and store parameters and state back with
 // 128-bit stores.  The ring keeps several tiles (about 160 KB per SM) in flight
