@@ -356,6 +356,67 @@ def time_oracle(items, params, min_seconds: float, max_passes: int):
     return params * passes / elapsed, used, passes, elapsed
 
 
+# ------------------------------------------------------------------ block-sharded arm
+
+def sharded_main(args, cfg, config, rank, local_rank, world, device):
+    """One workload over `world` ranks: every block is owned by one rank, the
+    W shards of a block are read in place from the worker ranks' exported
+    buffers (no collective in the path).  Total work is fixed: strong scaling."""
+    import torch.distributed as dist
+    from paper_2204_03211_b200 import sharded
+
+    def exchange(obj):
+        got = [None] * world
+        dist.all_gather_object(got, obj)
+        return got
+
+    red_dev = device if args.dist_backend == "nccl" else None
+    wl = sharded.ShardedWorkload(cfg, rank, world, local_rank, exchange, dist.barrier, param_device=device)
+    from paper_2204_03211_b200 import binding as B
+    wl.sh.svc.set_option(B.PS_OPT_OVERLAP, int(not args.in_stream))
+    wl.fill(0, device)
+    n_sched = max(1, min(args.warmup + args.steps, 8))
+    schedules = [configs.rounds_for(cfg, it, args.ticks) for it in range(n_sched)]
+    stream = torch.cuda.Stream(device)
+
+    def step(k, s):
+        n = wl.step(schedules[k % n_sched], s, key=k % n_sched)
+        if not args.in_stream:
+            wl.sh.svc.join(s)
+        return n
+
+    for k in range(args.warmup):
+        step(k, stream)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms, launches, host_ms = timed(lambda k, s: step(args.warmup + k, s), args.steps, stream, True, red_dev)
+    clocks = sampler.stop() if rank == 0 else {}
+    mine = [wl.owned_params, wl.owned_bytes, launches]
+    per_rank = exchange(mine)
+    if rank == 0:
+        value = cfg.num_params * args.steps / (ms * 1e-3)                     # every block once per step, all ranks
+        worst = max(r[1] for r in per_rank)
+        achieved = worst * args.steps / (ms * 1e-3) / 1e9                     # the most loaded rank's HBM traffic
+        peak, peak_kind = measured_peak()
+        config["parallelism"] = "blocks owned by %d ranks (longest-first partition), shards read in place from peers" % world
+        config["launch_mode"] = "in-stream" if args.in_stream else "overlapped, one ps_join per step"
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_source": peak_kind + " copy bandwidth",
+                         "note": "most loaded rank; with several GPUs the remote shards arrive over NVLink, "
+                                 "which bounds the step before HBM does"},
+            "per_rank": [{"params": r[0], "bytes_per_step": r[1], "launches": r[2]} for r in per_rank],
+            "cpu_baseline": None, "e2e": None, "gpu_launches": sum(r[2] for r in per_rank),
+            "host_ms_per_step": host_ms / args.steps, "clocks": clocks}))
+    wl.close()
+    dist.destroy_process_group()
+    return 0
+
+
 # ------------------------------------------------------------------ main
 
 def main():
@@ -378,6 +439,11 @@ def main():
     ap.add_argument("--in-stream", action="store_true",
                     help="enqueue every launch on the caller's stream (PS_OPT_OVERLAP = 0) instead of letting "
                          "the launches of a step overlap on the service's streams and joining once per step")
+    ap.add_argument("--shard-blocks", action="store_true",
+                    help="with --gpus N > 1: ONE workload whose blocks are owned by the N ranks (strong scaling; "
+                         "shards are read in place from the worker ranks' exported buffers) instead of N replicas")
+    ap.add_argument("--dist-backend", default="nccl", choices=["nccl", "gloo"],
+                    help="process-group backend for the barriers and the max over ranks")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -426,10 +492,16 @@ def main():
     dist_on = world > 1
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the aggregation path has no CPU fallback")
+    local_rank %= torch.cuda.device_count()
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     if dist_on:
-        dist.init_process_group("nccl", device_id=device)
+        if args.dist_backend == "nccl":
+            dist.init_process_group("nccl", device_id=device)
+        else:
+            dist.init_process_group("gloo")
+    if args.shard_blocks and dist_on:
+        return sharded_main(args, cfg, config, rank, local_rank, world, device)
 
     n_sched = max(1, min(args.warmup + args.steps, 8))
     wl = Workload(cfg, local_rank, args.ticks, n_sched, sparse=args.sparse_transport)

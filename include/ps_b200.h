@@ -317,6 +317,42 @@ int ps_aggregate_block_noalloc(const ps_job_desc* job, unsigned long long step, 
                                void* stream);
 
 /* ---------------------------------------------------------------------------
+ * Peer buffers: several Aggregators on the GPUs of one node.
+ *
+ * The paper spreads the tensors of a job over several Aggregator machines that
+ * exchange nothing but migrated tensors (Section 3.2).  On one node the
+ * counterpart is one service per GPU, one process each, every block owned by
+ * one of them; there is no collective in the aggregation path.  A worker's
+ * gradient shards then sit in another process's (often another GPU's) memory:
+ * the worker's process allocates them with ps_peer_alloc and passes the 64-byte
+ * handle to the owners by any host channel, an owner maps the buffer with
+ * ps_peer_open and gives the mapped address (plus the shard's offset) to
+ * ps_push.  The aggregation kernel reads it in place with ordinary loads: over
+ * NVLink when the GPUs differ, with no staging copy.
+ *
+ *   ps_peer_alloc  allocates `bytes` of device memory on `device` (its own
+ *                  allocation, 256-byte aligned) and writes its handle.
+ *                  Owner: the caller, until ps_peer_free.
+ *   ps_peer_open   maps a buffer exported by ANOTHER process into this one for
+ *                  use on `device` (peer access is enabled as needed); the
+ *                  mapping is read/write and stays valid until ps_peer_close or
+ *                  until the exporter frees the buffer, whichever comes first —
+ *                  the exporter must outlive every use.  Opening a handle in
+ *                  the process that exported it is an error (use the pointer).
+ * Errors: BAD_ARG, NOMEM, CUDA (text: ps_peer_last_error, per host thread).
+ * Ordering between the processes (the worker has finished writing a shard
+ * before the owner's launch reads it; the owner's launch has completed before
+ * the worker overwrites it) is the callers' business: a host barrier after a
+ * stream synchronize on each side is enough.
+ * ------------------------------------------------------------------------- */
+#define PS_PEER_HANDLE_BYTES 64
+int ps_peer_alloc(int device, size_t bytes, void** dev_ptr_out, unsigned char* handle_out);
+int ps_peer_free(int device, void* dev_ptr);
+int ps_peer_open(int device, const unsigned char* handle, void** dev_ptr_out);
+int ps_peer_close(int device, void* dev_ptr);
+const char* ps_peer_last_error(void);
+
+/* ---------------------------------------------------------------------------
  * Planner: which Aggregator (context) runs which aggregation task.  Host only.
  *
  * The paper's assignment heuristic — Section 3.3.1, Pseudocode 1 "Model

@@ -23,6 +23,7 @@ PS_ERR_TOO_LARGE = -9
 PS_NOALLOC_MAX_ELEMS = 1 << 24
 PS_DEVICE_NONE = -1
 PS_MAX_WORKERS = 256
+PS_PEER_HANDLE_BYTES = 64
 PS_OPT_CHUNK_ELEMS, PS_OPT_CTAS_PER_SM, PS_OPT_SORT_TASKS, PS_OPT_KERNEL, PS_OPT_PROFILE = 1, 2, 3, 4, 5
 PS_OPT_OVERLAP = 6
 PS_OPT_INLINE_TABLE = 7
@@ -98,6 +99,11 @@ _SIGNATURES = {
                                       C.POINTER(C.c_double)]),
     "ps_planner_num_aggregators": (C.c_int, [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
     "ps_planner_outlier_fits": (C.c_int, [C.c_double, C.c_double, C.c_double, C.c_double]),
+    "ps_peer_alloc": (C.c_int, [C.c_int, C.c_size_t, C.POINTER(C.c_void_p), C.c_char_p]),
+    "ps_peer_free": (C.c_int, [C.c_int, C.c_void_p]),
+    "ps_peer_open": (C.c_int, [C.c_int, C.c_char_p, C.POINTER(C.c_void_p)]),
+    "ps_peer_close": (C.c_int, [C.c_int, C.c_void_p]),
+    "ps_peer_last_error": (C.c_char_p, []),
     "ps_strerror": (C.c_char_p, [C.c_int]),
     "ps_last_cuda_error": (C.c_char_p, [C.c_void_p]),
     "ps_version": (C.c_char_p, []),
@@ -430,6 +436,35 @@ class Service:
         m = _Mem()
         m.__cuda_array_interface__ = {"shape": (nelem,), "typestr": "<f4", "data": (ptr, False), "version": 2}
         return torch.as_tensor(m, device="cuda" if device is None else "cuda:%d" % device)
+
+
+def _check_peer(rc: int, where: str):
+    if rc != PS_OK:
+        raise PsError(rc, where, load().ps_peer_last_error().decode() if rc == PS_ERR_CUDA else "")
+
+
+def ps_peer_alloc(device: int, nbytes: int):
+    """Returns (device pointer, 64-byte handle) of a buffer other processes can map."""
+    out, handle = C.c_void_p(), C.create_string_buffer(PS_PEER_HANDLE_BYTES)
+    _check_peer(load().ps_peer_alloc(device, nbytes, C.byref(out), handle), "ps_peer_alloc")
+    return out.value, handle.raw
+
+
+def ps_peer_free(device: int, ptr: int):
+    _check_peer(load().ps_peer_free(device, ptr), "ps_peer_free")
+
+
+def ps_peer_open(device: int, handle: bytes) -> int:
+    """Maps a buffer exported by another process; returns its address here."""
+    if len(handle) != PS_PEER_HANDLE_BYTES:
+        raise PsError(PS_ERR_BAD_ARG, "ps_peer_open", "handle must be %d bytes" % PS_PEER_HANDLE_BYTES)
+    out = C.c_void_p()
+    _check_peer(load().ps_peer_open(device, handle, C.byref(out)), "ps_peer_open")
+    return out.value
+
+
+def ps_peer_close(device: int, ptr: int):
+    _check_peer(load().ps_peer_close(device, ptr), "ps_peer_close")
 
 
 def _bind(name):

@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libps_b200.so")
-SOURCES = [os.path.join(CSRC, "ps_service.cu"), os.path.join(CSRC, "ps_planner.cpp")]
+SOURCES = [os.path.join(CSRC, "ps_service.cu"), os.path.join(CSRC, "ps_planner.cpp"), os.path.join(CSRC, "ps_peer.cpp")]
 
 
 def _deps():

@@ -1,0 +1,250 @@
+"""Block-sharded deployment: several Aggregators on the GPUs of one node.
+
+The paper spreads the tensors of a job over several Aggregators, which exchange
+nothing with one another except migrated tensors (Section 3.2; aggregation
+tasks are independent per tensor, Section 2.2).  Here one process per GPU runs
+one service; every (job, block) has ONE owner rank, which holds its master copy
+and runs its aggregation.  There is no collective in the aggregation path: the
+W gradient shards of a block sit in buffers that the workers' processes export
+(`ps_peer_alloc`), the owner maps them (`ps_peer_open`) and pushes the mapped
+addresses, and the aggregation kernel reads them in place — through NVLink when
+the worker's GPU is not the owner's.
+
+This module is host logic only (who owns what, which address a shard has in
+which process); every arithmetic step runs in the library's kernels.
+"""
+from __future__ import annotations
+
+from . import binding as B
+
+
+def partition(costs: dict, world: int) -> dict:
+    """Owner rank of every key of `costs` ({(job, block): cost}, cost = bytes the
+    block's aggregation moves).  Longest-processing-time greedy: heaviest block
+    first, to the least-loaded rank, lowest rank on ties; keys break cost ties.
+    Deterministic, so every rank computes the same map without communicating.
+    The heaviest rank carries at most 4/3 of the optimum (Graham's bound)."""
+    if world < 1:
+        raise ValueError("world must be >= 1")
+    load = [0.0] * world
+    owner = {}
+    for key in sorted(costs, key=lambda k: (-costs[k], k)):
+        r = min(range(world), key=lambda i: (load[i], i))
+        owner[key] = r
+        load[r] += costs[key]
+    return owner
+
+
+def worker_rank(worker: int, world: int) -> int:
+    """Rank whose process holds worker w's shards (workers dealt round-robin)."""
+    return worker % world
+
+
+class PeerSlabs:
+    """One exported device buffer per rank, mapped by every other rank.
+
+    `exchange(obj) -> list` is an all-gather of a picklable object over the
+    ranks (e.g. `torch.distributed.all_gather_object`).  `base[r]` is the
+    address of rank r's buffer in THIS process (its own buffer: the pointer
+    itself).  A rank that needs no buffer passes nbytes = 0."""
+
+    def __init__(self, rank: int, world: int, device: int, nbytes: int, exchange):
+        self.rank, self.world, self.device = rank, world, device
+        self.own, handle = (B.ps_peer_alloc(device, nbytes) if nbytes > 0 else (0, b""))
+        self.nbytes = nbytes
+        handles = exchange(handle)
+        if len(handles) != world:
+            raise ValueError("exchange returned %d handles for %d ranks" % (len(handles), world))
+        self.base, self._opened = [0] * world, []
+        for r, h in enumerate(handles):
+            if r == rank:
+                self.base[r] = self.own
+            elif h:
+                self.base[r] = B.ps_peer_open(device, h)
+                self._opened.append(self.base[r])
+
+    def close(self):
+        """Unmaps the peers' buffers and frees this rank's own.  Call it on every
+        rank only after all ranks have finished using the buffers."""
+        for p in self._opened:
+            B.ps_peer_close(self.device, p)
+        self._opened = []
+        if self.own:
+            B.ps_peer_free(self.device, self.own)
+            self.own = 0
+
+
+class ShardedService:
+    """The local service of one rank plus the ownership map.
+
+    Jobs are registered on every rank in the same order (hyper-parameters are a
+    few bytes); a block is registered only in its owner's service.  push /
+    aggregate / pull act on owned blocks and ignore the others, so every rank can
+    run the same loop over the whole ready list."""
+
+    def __init__(self, rank: int, world: int, device: int, num_contexts: int = 1, arena_bytes: int = 1 << 30):
+        self.rank, self.world, self.device = rank, world, device
+        self.svc = B.Service(device, num_contexts, arena_bytes)
+        self.owner = {}
+
+    def close(self):
+        self.svc.close()
+
+    def register_job(self, **hp) -> int:
+        return self.svc.register_job(**hp)
+
+    def set_owners(self, owner: dict):
+        self.owner = dict(owner)
+
+    def owns(self, job: int, block: int) -> bool:
+        return self.owner[(job, block)] == self.rank
+
+    def register_block(self, job: int, block: int, nelem: int, ctx: int = 0, init=None) -> bool:
+        if not self.owns(job, block):
+            return False
+        self.svc.register_block(job, block, nelem, ctx, init)
+        return True
+
+    def push(self, job: int, block: int, worker: int, ptr) -> bool:
+        """`ptr`: the shard's address in THIS process (a mapped peer address or a
+        local one)."""
+        if not self.owns(job, block):
+            return False
+        self.svc.push(job, block, worker, ptr)
+        return True
+
+    def owned(self, ready) -> list:
+        return [(j, b) for (j, b) in ready if self.owns(j, b)]
+
+    def aggregate(self, ready, stream=None) -> int:
+        """One packed launch for the owned tasks of `ready`; returns how many."""
+        mine = self.owned(ready)
+        if mine:
+            self.svc.aggregate(mine, stream)
+        return len(mine)
+
+    def pull(self, job: int, block: int) -> int:
+        if not self.owns(job, block):
+            raise B.PsError(B.PS_ERR_BAD_ARG, "ShardedService.pull", "block (%d,%d) is owned by rank %d" % (
+                job, block, self.owner[(job, block)]))
+        return self.svc.pull(job, block)
+
+
+def device_bytes(ptr: int, nbytes: int, device: int):
+    """uint8 torch view of device memory that torch did not allocate (no copy)."""
+    import torch
+
+    class _Mem:
+        pass
+
+    m = _Mem()
+    m.__cuda_array_interface__ = {"shape": (nbytes,), "typestr": "|u1", "data": (ptr, False), "version": 2}
+    return torch.as_tensor(m, device="cuda:%d" % device)
+
+
+class ShardedWorkload:
+    """A benchmark configuration (workload.configs.Config) run block-sharded.
+
+    Rank r owns the blocks `partition` gives it and, as a worker host, holds the
+    gradient shards of workers w with w mod world == r of EVERY job in one
+    exported buffer: job after job, worker after worker, each shard row padded
+    to 128 elements.  Every rank can compute every rank's layout, so only the
+    64-byte handles travel.  `exchange` as in PeerSlabs; `barrier()` blocks
+    until every rank has called it."""
+
+    ROW_ALIGN = 128
+
+    def __init__(self, cfg, rank: int, world: int, device: int, exchange, barrier, arena_slack: int = 64 << 20,
+                 param_device="cpu"):
+        import numpy as np
+        from workload import configs, generate
+        self.cfg, self.rank, self.world, self.device = cfg, rank, world, device
+        self.barrier = barrier
+        self._generate, self._np = generate, np
+        costs = {(j, b.block): job.bytes_per_elem() * b.nelem for j, job in enumerate(cfg.jobs) for b in job.blocks}
+        owner = partition(costs, world)
+        mine = [(j, b) for j, job in enumerate(cfg.jobs) for b in job.blocks if owner[(j, b.block)] == rank]
+        arena = sum(3 * (4 * b.nelem + 256) for _, b in mine) + arena_slack
+        self.sh = ShardedService(rank, world, device, cfg.num_contexts, arena)
+        self.sh.set_owners(owner)
+        self.owned_params = sum(b.nelem for _, b in mine)
+        self.owned_bytes = sum(costs[(j, b.block)] for j, b in mine)
+        # layout of every rank's exported buffer
+        self.row_off = {}                       # (job, worker) -> byte offset inside its host rank's buffer
+        size = [0] * world
+        for j, job in enumerate(cfg.jobs):
+            esz = 2 if job.grad_dtype == configs.BF16 else 4
+            row = (job.num_params + self.ROW_ALIGN - 1) // self.ROW_ALIGN * self.ROW_ALIGN * esz
+            for w in range(job.num_workers):
+                r = worker_rank(w, world)
+                self.row_off[(j, w)] = size[r]
+                size[r] += row
+        self.slabs = PeerSlabs(rank, world, device, size[rank], exchange)
+        for j, job in enumerate(cfg.jobs):
+            assert self.sh.register_job(**job.hparams()) == j
+            p0 = generate.init_params(cfg, j, param_device)     # the seeded generator of that device kind
+            for b in job.blocks:
+                if owner[(j, b.block)] == rank:
+                    self.sh.register_block(j, b.block, b.nelem, configs.initial_context(cfg, j, b.block),
+                                           p0[b.job_offset:b.job_offset + b.nelem].contiguous())
+            del p0
+        self._args = {}
+
+    def close(self):
+        import torch
+        torch.cuda.synchronize(self.device)
+        self.barrier()                          # nobody reads a peer's buffer any more
+        self.slabs.close()
+        self.sh.close()
+
+    def shard_address(self, job: int, block: int, worker: int) -> int:
+        """Address, in this process, of worker w's shard of (job, block)."""
+        spec = self.cfg.jobs[job]
+        esz = 2 if spec.grad_dtype == 1 else 4
+        return (self.slabs.base[worker_rank(worker, self.world)] + self.row_off[(job, worker)]
+                + spec.blocks[block].job_offset * esz)
+
+    def fill(self, iteration: int, gen_device="cpu"):
+        """Writes this rank's workers' gradients of `iteration` into its exported
+        buffer (the seeded generator's values, identical to the unsharded run
+        that generates on the same kind of device), then meets the other ranks:
+        on return every rank's buffer is complete."""
+        import torch
+        dev = torch.device("cuda", self.device)
+        for j, job in enumerate(self.cfg.jobs):
+            slab = self._generate.grad_slab(self.cfg, j, iteration, gen_device)
+            rowbytes = job.num_params * slab.element_size()
+            for w in range(job.num_workers):
+                if worker_rank(w, self.world) != self.rank:
+                    continue
+                dst = device_bytes(self.slabs.own + self.row_off[(j, w)], rowbytes, self.device)
+                dst.copy_(slab[w].contiguous().view(torch.uint8).to(dev))      # no-op move when generated on dev
+            del slab
+        torch.cuda.synchronize(dev)
+        self.barrier()
+
+    def _round_args(self, key, ready):
+        if key not in self._args:
+            np = self._np
+            mine = self.sh.owned(ready)
+            jobs, blocks, workers, ptrs = [], [], [], []
+            for (j, b) in mine:
+                for w in range(self.cfg.jobs[j].num_workers):
+                    jobs.append(j); blocks.append(b); workers.append(w)
+                    ptrs.append(self.shard_address(j, b, w))
+            self._args[key] = (mine, np.array(jobs, np.int32), np.array(blocks, np.int32),
+                               np.array(workers, np.int32), np.array(ptrs, np.uint64), B.make_tasks(mine))
+        return self._args[key]
+
+    def step(self, rounds, stream=None, key=0) -> int:
+        """Push and aggregate this rank's blocks of every round; returns launches.
+        `key` names the schedule so that call arguments are built once."""
+        launches = 0
+        for i, ready in enumerate(rounds):
+            mine, jobs, blocks, workers, ptrs, tasks = self._round_args((key, i), ready)
+            if not mine:
+                continue
+            self.sh.svc.push_batch(jobs, blocks, workers, ptrs)
+            self.sh.svc.aggregate(tasks, stream)
+            launches += 1
+        return launches
