@@ -316,6 +316,37 @@ int ps_aggregate_block_noalloc(const ps_job_desc* job, unsigned long long step, 
                                const void* const* shard_dev_ptrs, double* sqnorm_dev_out_or_null,
                                void* stream);
 
+/* Migration between two services (the paper's migration between Aggregator
+ * machines, Section 3.2 and Appendix B: the old Aggregator copies the tensor's
+ * contents and metadata to the new one, which must not update the tensor before
+ * the copy has landed).  ps_migrate_block moves a block between contexts of ONE
+ * service; these three calls move it between services, e.g. between the GPUs of
+ * a block-sharded deployment, through any device memory both can address (a
+ * peer buffer):
+ *
+ *   ps_block_export  enqueues on `stream`, after the block's last aggregate, a
+ *       copy of its packed state into dst_dev: parameters | state0 | (state1),
+ *       each section round_up(4*nelem, 256) bytes — *bytes_out in total — and
+ *       reports the block's step counter.  dst_dev == NULL only reports the two
+ *       numbers.  The service is unchanged; pending pushes are not exported.
+ *   ps_block_import  for a block registered here (same nelem, same optimizer):
+ *       enqueues on `stream` the copy of such a packed state into the block's
+ *       range and sets its step counter.  Later aggregates of the block wait for
+ *       the copy (they are ordered after it whatever their stream); pushes may
+ *       arrive meanwhile.  src_bytes must equal the block's packed size.
+ *   ps_unregister_block  waits (host) for the work this service enqueued for
+ *       the block, releases its arena range and staging buffer and forgets the
+ *       id, which may be registered again.  Pending pushes are dropped.
+ * The caller orders the two sides: the export's stream has reached the copy's
+ * end before the importer's copy starts (same process: an event; two
+ * processes: synchronize, then a host barrier).
+ * Errors: BAD_ARG (unknown block, dst too small, size mismatch), NO_DEVICE, CUDA. */
+int ps_block_export(ps_service* svc, int job, int block, void* dst_dev, size_t dst_cap, size_t* bytes_out,
+                    unsigned long long* step_out, void* stream);
+int ps_block_import(ps_service* svc, int job, int block, const void* src_dev, size_t src_bytes,
+                    unsigned long long step, void* stream);
+int ps_unregister_block(ps_service* svc, int job, int block);
+
 /* ---------------------------------------------------------------------------
  * Peer buffers: several Aggregators on the GPUs of one node.
  *

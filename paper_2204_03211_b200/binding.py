@@ -99,6 +99,10 @@ _SIGNATURES = {
                                       C.POINTER(C.c_double)]),
     "ps_planner_num_aggregators": (C.c_int, [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
     "ps_planner_outlier_fits": (C.c_int, [C.c_double, C.c_double, C.c_double, C.c_double]),
+    "ps_block_export": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t),
+                                 C.POINTER(C.c_ulonglong), C.c_void_p]),
+    "ps_block_import": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_ulonglong, C.c_void_p]),
+    "ps_unregister_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int]),
     "ps_peer_alloc": (C.c_int, [C.c_int, C.c_size_t, C.POINTER(C.c_void_p), C.c_char_p]),
     "ps_peer_free": (C.c_int, [C.c_int, C.c_void_p]),
     "ps_peer_open": (C.c_int, [C.c_int, C.c_char_p, C.POINTER(C.c_void_p)]),
@@ -438,6 +442,24 @@ class Service:
         return torch.as_tensor(m, device="cuda" if device is None else "cuda:%d" % device)
 
 
+def ps_block_export(svc, job: int, block: int, dst=None, dst_cap: int = 0, stream=None):
+    """Returns (packed bytes, step).  With dst (device tensor or address) also
+    enqueues the copy of the block's packed state into it."""
+    n, step = C.c_size_t(), C.c_ulonglong()
+    _check(load().ps_block_export(svc, job, block, _ptr(dst), dst_cap, C.byref(n), C.byref(step),
+                                  _stream_ptr(stream)), "ps_block_export", svc)
+    return n.value, step.value
+
+
+def ps_block_import(svc, job: int, block: int, src, src_bytes: int, step: int, stream=None):
+    _check(load().ps_block_import(svc, job, block, _ptr(src), src_bytes, step, _stream_ptr(stream)),
+           "ps_block_import", svc)
+
+
+def ps_unregister_block(svc, job: int, block: int):
+    _check(load().ps_unregister_block(svc, job, block), "ps_unregister_block", svc)
+
+
 def _check_peer(rc: int, where: str):
     if rc != PS_OK:
         raise PsError(rc, where, load().ps_peer_last_error().decode() if rc == PS_ERR_CUDA else "")
@@ -480,5 +502,5 @@ def _bind(name):
 
 for _n in ("register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "aggregate", "join", "pull", "pull_batch", "pull_host",
            "migrate_block", "migrate_blocks", "block_stats", "block_profile", "job_profile", "block_state", "plan", "set_option", "get_option", "arena_info",
-           "launch_info", "device_status"):
+           "launch_info", "device_status", "block_export", "block_import", "unregister_block"):
     setattr(Service, _n, _bind(_n))

@@ -622,6 +622,9 @@ int ps_register_block(ps_service* s, int job, int block, size_t nelem, int ctx, 
       char* base = s->ctxs[ctx].base + b.off;
       e = cudaMemset(base, 0, b.bytes);
       if (e == cudaSuccess && init) e = cudaMemcpy(base, init, nelem * sizeof(float), cudaMemcpyDefault);
+      // a device memset may return before it has run, and the service's streams do not
+      // synchronize with the default stream: wait here, once per registration
+      if (e == cudaSuccess) e = cudaStreamSynchronize(cudaStreamLegacy);
       if (e != cudaSuccess) { s->cuda_err = cudaGetErrorString(e); rc = PS_ERR_CUDA; }
     }
     if (rc) { s->ctxs[ctx].arena.release(b.off, b.bytes); return rc; }
@@ -922,6 +925,23 @@ int ps_pull_host(ps_service* s, int job, int block, float* dst, void* stream_) {
   return PS_OK;
 }
 
+// A copy batch that is not in use (its event exists on return).
+static int free_batch(ps_service* s, int* out) {
+  int batch = -1;
+  for (int i = 0; i < (int)s->batches.size(); ++i)
+    if (!s->batches[i].pending) { batch = i; break; }
+  if (batch < 0) {
+    s->batches.emplace_back();
+    batch = (int)s->batches.size() - 1;
+  }
+  if (!s->batches[batch].ev) {
+    cudaError_t e = cudaEventCreateWithFlags(&s->batches[batch].ev, cudaEventDisableTiming);
+    if (e != cudaSuccess) { s->cuda_err = cudaGetErrorString(e); return PS_ERR_CUDA; }
+  }
+  *out = batch;
+  return PS_OK;
+}
+
 // Moves the listed blocks (indices into s->blocks) to dst_ctx as ONE batch: all
 // destination ranges are reserved first (nothing changes if one does not fit),
 // the copies are ordered after each block's last aggregate and last move, one
@@ -946,15 +966,9 @@ static int migrate_many(ps_service* s, const std::vector<int>& bis, int dst_ctx,
     for (auto& m : moves) s->ctxs[dst_ctx].arena.release(m.noff, s->blocks[m.bi].bytes);
   };
   int batch = -1;
-  for (int i = 0; i < (int)s->batches.size(); ++i)
-    if (!s->batches[i].pending) { batch = i; break; }
-  if (batch < 0) {
-    s->batches.emplace_back();
-    batch = (int)s->batches.size() - 1;
-  }
-  if (!s->batches[batch].ev) {
-    cudaError_t e = cudaEventCreateWithFlags(&s->batches[batch].ev, cudaEventDisableTiming);
-    if (e != cudaSuccess) { undo(); s->cuda_err = cudaGetErrorString(e); return PS_ERR_CUDA; }
+  {
+    int rc = free_batch(s, &batch);
+    if (rc) { undo(); return rc; }
   }
   unsigned int waited = 0;
   for (auto& m : moves) {
@@ -1029,6 +1043,94 @@ int ps_migrate_blocks(ps_service* s, const ps_task* tasks, int n, int dst_ctx, v
   PS_CUDA(s, cudaSetDevice(s->device));
   ++s->call_id;
   return migrate_many(s, bis, dst_ctx, static_cast<cudaStream_t>(stream_));
+}
+
+// Marks `stream`'s position as a copy batch of block b: later work on b waits for it.
+static int mark_copy(ps_service* s, Block& b, cudaStream_t stream) {
+  int batch = -1;
+  int rc = free_batch(s, &batch);
+  if (rc) return rc;
+  PS_CUDA(s, cudaEventRecord(s->batches[batch].ev, stream));
+  MigBatch& mb = s->batches[batch];
+  mb.pending = true;
+  mb.seen_call = mb.waited_call = 0;
+  b.mig_batch = batch;
+  return PS_OK;
+}
+
+int ps_block_export(ps_service* s, int job, int block, void* dst_dev, size_t dst_cap, size_t* bytes_out,
+                    unsigned long long* step_out, void* stream_) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  const int bi = find_block(s, job, block);
+  if (bi < 0) return PS_ERR_BAD_ARG;
+  Block& b = s->blocks[bi];
+  if (bytes_out) *bytes_out = b.bytes;
+  if (step_out) *step_out = b.step;
+  if (!dst_dev) return PS_OK;                       // size query
+  if (dst_cap < b.bytes) return PS_ERR_BAD_ARG;
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  PS_CUDA(s, cudaSetDevice(s->device));
+  ++s->call_id;
+  int rc = order_after_block(s, b, stream);
+  if (rc) return rc;
+  PS_CUDA(s, cudaMemcpyAsync(dst_dev, s->ctxs[b.ctx].base + b.off, b.bytes, cudaMemcpyDefault, stream));
+  return mark_copy(s, b, stream);
+}
+
+int ps_block_import(ps_service* s, int job, int block, const void* src_dev, size_t src_bytes,
+                    unsigned long long step, void* stream_) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  const int bi = find_block(s, job, block);
+  if (bi < 0 || !src_dev) return PS_ERR_BAD_ARG;
+  Block& b = s->blocks[bi];
+  if (src_bytes != b.bytes) return PS_ERR_BAD_ARG;
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  PS_CUDA(s, cudaSetDevice(s->device));
+  ++s->call_id;
+  int rc = order_after_block(s, b, stream);
+  if (rc) return rc;
+  PS_CUDA(s, cudaMemcpyAsync(s->ctxs[b.ctx].base + b.off, src_dev, b.bytes, cudaMemcpyDefault, stream));
+  rc = mark_copy(s, b, stream);
+  if (rc) return rc;
+  b.step = step;
+  return PS_OK;
+}
+
+int ps_unregister_block(ps_service* s, int job, int block) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  const int bi = find_block(s, job, block);
+  if (bi < 0) return PS_ERR_BAD_ARG;
+  Block& b = s->blocks[bi];
+  if (has_device(s)) {
+    PS_CUDA(s, cudaSetDevice(s->device));
+    ++s->call_id;
+    // everything this service enqueued for the block: its last launch, its last copy
+    if (b.last_slot >= 0) {
+      Slot& sl = s->slots[b.last_slot];
+      if (sl.inflight && sl.gen == b.last_slot_gen) PS_CUDA(s, cudaEventSynchronize(sl.done));
+    }
+    if (b.mig_batch >= 0) {
+      bool ready = false;
+      int rc = batch_ready(s, b.mig_batch, true, &ready);
+      if (rc) return rc;
+      b.mig_batch = -1;
+    }
+    if (b.staging) {
+      PS_CUDA(s, cudaFree(b.staging));
+      b.staging = nullptr;
+    }
+  }
+  s->ctxs[b.ctx].arena.release(b.off, b.bytes);
+  s->jobs[b.job].block_of_id[b.id] = -1;
+  b.nelem = 0;
+  b.bytes = 0;
+  b.npushed = 0;
+  return PS_OK;
 }
 
 int ps_block_stats(ps_service* s, int job, int block, double* sq_out, unsigned long long* step_out) {

@@ -10,6 +10,10 @@ W gradient shards of a block sit in buffers that the workers' processes export
 addresses, and the aggregation kernel reads them in place — through NVLink when
 the worker's GPU is not the owner's.
 
+A block changes owner by a migration between services (`ShardedWorkload.migrate`:
+ps_block_export into an exported buffer, ps_block_import on the new owner,
+ps_unregister_block on the old one).
+
 This module is host logic only (who owns what, which address a shard has in
 which process); every arithmetic step runs in the library's kernels.
 """
@@ -222,6 +226,65 @@ class ShardedWorkload:
             del slab
         torch.cuda.synchronize(dev)
         self.barrier()
+
+    def packed_bytes(self, job: int, block: int) -> int:
+        """Size of a block's packed state (parameters and optimizer state, each
+        section rounded up to 256 bytes): what a migration moves."""
+        spec = self.cfg.jobs[job]
+        sec = (4 * spec.blocks[block].nelem + 255) // 256 * 256
+        return sec * (3 if spec.opt == 1 else 2)
+
+    def migrate(self, moves, exchange, stream=None):
+        """Changes the owner of blocks: moves = [(job, block, new_rank)], the
+        same list on every rank (a collective call, like a migration ordered by
+        the paper's pMaster).  The old owner copies the block's packed state into
+        a buffer it exports, the new owner registers the block and copies it in
+        from its mapping of that buffer, then the old owner forgets the block.
+        Aggregates of a moved block that the new owner enqueues afterwards wait
+        for the copy.  The new owner's arena must have room for the block
+        (`arena_slack` at construction) before the old owner releases its range.
+        Returns the bytes this rank sent."""
+        import torch
+        moves = [(j, b, r) for (j, b, r) in moves if self.sh.owner[(j, b)] != r]
+        out = [(j, b, r) for (j, b, r) in moves if self.sh.owner[(j, b)] == self.rank]
+        size = sum(self.packed_bytes(j, b) for j, b, _ in out)
+        lane = PeerSlabs(self.rank, self.world, self.device, size, exchange)
+        offs, off_by_rank = {}, [0] * self.world
+        for (j, b, r) in moves:                        # every rank derives every offset
+            src = self.sh.owner[(j, b)]
+            offs[(j, b)] = off_by_rank[src]
+            off_by_rank[src] += self.packed_bytes(j, b)
+        steps = {}
+        for (j, b, r) in out:
+            n = self.packed_bytes(j, b)
+            got, step = self.sh.svc.block_export(j, b, lane.own + offs[(j, b)], n, stream)
+            assert got == n
+            steps[(j, b)] = step
+        torch.cuda.synchronize(self.device)            # the exported copies have landed ...
+        all_steps = {}
+        for d in exchange(steps):                      # ... and this exchange is the barrier that says so
+            all_steps.update(d)
+        for (j, b, r) in moves:
+            if r != self.rank:
+                continue
+            src = self.sh.owner[(j, b)]
+            spec = self.cfg.jobs[j]
+            self.sh.owner[(j, b)] = r
+            self.sh.svc.register_block(j, b, spec.blocks[b].nelem, 0, None)
+            self.sh.svc.block_import(j, b, lane.base[src] + offs[(j, b)], self.packed_bytes(j, b),
+                                     all_steps[(j, b)], stream)
+        torch.cuda.synchronize(self.device)            # the imports have read the lanes
+        self.barrier()
+        for (j, b, r) in out:
+            self.sh.svc.unregister_block(j, b)
+        for (j, b, r) in moves:
+            self.sh.owner[(j, b)] = r
+        lane.close()
+        self._args.clear()
+        self.owned_params = sum(self.cfg.jobs[j].blocks[b].nelem for (j, b), r in self.sh.owner.items() if r == self.rank)
+        self.owned_bytes = sum(self.cfg.jobs[j].bytes_per_elem() * self.cfg.jobs[j].blocks[b].nelem
+                               for (j, b), r in self.sh.owner.items() if r == self.rank)
+        return size
 
     def _round_args(self, key, ready):
         if key not in self._args:

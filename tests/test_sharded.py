@@ -5,8 +5,9 @@ CPU: the ownership map (balanced, deterministic, identical on every rank) and
 the per-rank registry, with two gloo ranks over planning-only services.
 GPU: two processes sharing one device, each the owner of half the blocks and
 the host of half the workers; shards are read in place from the other
-process's exported buffer (CUDA IPC) and every owned block is compared bit for
-bit with the CPU oracle.  The two ranks' kernels never wait on one another:
+process's exported buffer (CUDA IPC), blocks change owner between two
+iterations (export, import, unregister) and every owned block is compared bit
+for bit with the CPU oracle.  The two ranks' kernels never wait on one another:
 the ranks meet only in host barriers."""
 import json
 import os
@@ -129,30 +130,41 @@ def _gpu_rank(rank, world, port, out):
 
     a = tiny_config([70001, 5, 4096, 300000, 33], 3).jobs[0]
     b = tiny_config([1 << 18, 12289, 1, 8192], 4, opt=configs.ADAM, grad_dtype=configs.BF16).jobs[0]
-    cfg = configs.Config("sharded-tiny", 321, 2, [a, b])
-    wl = sharded.ShardedWorkload(cfg, rank, world, 0, exchange, dist.barrier, arena_slack=1 << 20)
+    cfg = configs.Config("sharded-tiny", 321, 3, [a, b])
+    wl = sharded.ShardedWorkload(cfg, rank, world, 0, exchange, dist.barrier, arena_slack=16 << 20)   # room for adopted blocks
+    # the oracle of each rank follows EVERY block (they are tiny), so that a block
+    # adopted by this rank half-way has its history
     ora = A.OracleAggregator(1, 0)
     for j, job in enumerate(cfg.jobs):
         assert ora.register_job(oracle_hp(job)) == j
         p0 = generate.init_params(cfg, j)
         for blk in job.blocks:
-            if wl.sh.owns(j, blk.block):
-                ora.register_block(j, blk.block, blk.nelem, 0, p0[blk.job_offset:blk.job_offset + blk.nelem].numpy())
+            ora.register_block(j, blk.block, blk.nelem, 0, p0[blk.job_offset:blk.job_offset + blk.nelem].numpy())
     every = configs.rounds_all(cfg)[0]
     rounds = [every[:4], every[4:]]
-    remote_reads = 0
-    for it in range(2):
+    remote_reads, adopted, sent = 0, set(), 0
+    for it in range(3):
+        if it == 2:
+            # between two iterations every rank hands its two lowest blocks of each job to the other rank
+            owner0 = dict(wl.sh.owner)
+            moves = []
+            for r in range(world):
+                for j in range(len(cfg.jobs)):
+                    theirs = sorted(blk for (jj, blk), o in owner0.items() if jj == j and o == r)
+                    moves += [(j, blk, 1 - r) for blk in theirs[:2]]
+            before = set(wl.sh.owned(every))
+            sent = wl.migrate(moves, exchange)
+            adopted = set(wl.sh.owned(every)) - before
         wl.fill(it, "cpu")
         assert wl.step(rounds, key=0) >= 1
         for j, job in enumerate(cfg.jobs):
             host = to_np(generate.grad_slab(cfg, j, it))
             for blk in job.blocks:
-                if not wl.sh.owns(j, blk.block):
-                    continue
                 for w in range(job.num_workers):
                     ora.push(j, blk.block, w, host[w, blk.job_offset:blk.job_offset + blk.nelem])
-                    remote_reads += int(sharded.worker_rank(w, world) != rank)
-        ora.aggregate(wl.sh.owned(every))
+                    if wl.sh.owns(j, blk.block):
+                        remote_reads += int(sharded.worker_rank(w, world) != rank)
+        ora.aggregate(every)
         torch.cuda.synchronize()
         dist.barrier()                                             # every rank has read the buffers: refill allowed
     ok, checked = True, 0
@@ -167,11 +179,18 @@ def _gpu_rank(rank, world, port, out):
             ok &= np.array_equal(wl.sh.svc.view(s1, n).cpu().numpy(), rv)
         sq, step = wl.sh.svc.block_stats(j, blk)
         rsq, rstep = ora.block_stats(j, blk)
-        ok &= step == rstep == 2 and abs(sq - rsq) <= 1e-5 * abs(rsq) + 1e-300
+        ok &= step == rstep == 3 and abs(sq - rsq) <= 1e-5 * abs(rsq) + 1e-300
         checked += 1
+    gone = [k for k in every if not wl.sh.owns(*k)]
+    for (j, blk) in gone[:2]:                                      # a block that left is unknown here
+        try:
+            wl.sh.svc.pull(j, blk)
+            ok = False
+        except B.PsError as e:
+            ok &= e.status == B.PS_ERR_BAD_ARG
     with open(out % rank, "w") as f:
-        json.dump({"ok": bool(ok), "checked": checked, "remote_reads": remote_reads,
-                   "status": wl.sh.svc.device_status()}, f)
+        json.dump({"ok": bool(ok), "checked": checked, "remote_reads": remote_reads, "adopted": len(adopted),
+                   "sent": sent, "status": wl.sh.svc.device_status()}, f)
     wl.close()
     dist.barrier()
     dist.destroy_process_group()
@@ -185,6 +204,7 @@ def test_two_processes_on_one_device_read_each_others_shards_in_place(tmp_path):
     assert all(g["ok"] and g["status"] == 0 for g in got), got
     assert sum(g["checked"] for g in got) == 9 and min(g["checked"] for g in got) >= 2
     assert all(g["remote_reads"] > 0 for g in got)                 # each rank consumed shards hosted by the other
+    assert all(g["adopted"] >= 2 and g["sent"] > 0 for g in got)   # and blocks changed owner in both directions
 
 
 @pytest.mark.gpu
@@ -200,3 +220,94 @@ def test_bench_block_sharded_arm_two_ranks_on_one_device():
     assert line["n_gpus"] == 2 and line["scaling"] == "strong" and line["value"] > 0
     assert sum(p["params"] for p in line["per_rank"]) == cfg.num_params
     assert line["gpu_launches"] == sum(p["launches"] for p in line["per_rank"]) == 2 * 5
+
+
+def test_unregister_and_export_query_on_a_planning_only_service():
+    svc = B.Service(device=B.PS_DEVICE_NONE, num_contexts=1, arena_bytes_per_ctx=1 << 20)
+    try:
+        j = svc.register_job(opt=B.PS_ADAM, grad_dtype=B.PS_F32, num_workers=2, lr=1e-3)
+        svc.register_block(j, 3, 1000, 0, None)
+        used = svc.arena_info(0)[0]
+        assert used == 3 * 4096                                    # p | m | v, each 4000 B rounded up to 256
+        assert svc.block_export(j, 3) == (3 * 4096, 0)             # size query: no device needed
+        with pytest.raises(B.PsError) as e:
+            svc.block_export(j, 3, 1 << 20, 3 * 4096)
+        assert e.value.status == B.PS_ERR_NO_DEVICE
+        with pytest.raises(B.PsError) as e:
+            svc.block_export(j, 3, 1 << 20, 100)                   # destination too small
+        assert e.value.status == B.PS_ERR_BAD_ARG
+        with pytest.raises(B.PsError) as e:
+            svc.block_import(j, 3, 1 << 20, 17, 5)                 # not the block's packed size
+        assert e.value.status == B.PS_ERR_BAD_ARG
+        svc.unregister_block(j, 3)
+        assert svc.arena_info(0)[0] == 0
+        for call in (lambda: svc.unregister_block(j, 3), lambda: svc.block_export(j, 3),
+                     lambda: svc.push(j, 3, 0, np.zeros(4, np.float32))):
+            with pytest.raises(B.PsError) as e:
+                call()
+            assert e.value.status == B.PS_ERR_BAD_ARG
+        svc.register_block(j, 3, 500, 0, None)                     # the id can be used again
+        assert svc.block_export(j, 3) == (3 * 2048, 0)
+    finally:
+        svc.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("opt,dt", [(configs.SGD, configs.F32), (configs.ADAM, configs.BF16)])
+def test_block_moves_between_two_services_and_training_continues_bit_for_bit(opt, dt):
+    """Two services on one device stand for two Aggregators.  A block trains two
+    iterations on the first, moves (export -> import -> unregister) and trains
+    two more on the second: parameters, state and the step counter (Adam's bias
+    correction depends on it) must equal the oracle's four uninterrupted
+    iterations."""
+    from helpers import Pair, tiny_config, to_np
+    from workload import generate
+    cfg = tiny_config([70001, 4096], 3, opt=opt, grad_dtype=dt)
+    pair = Pair(cfg)
+    other = B.Service(0, 1, 8 << 20)
+    try:
+        job = cfg.jobs[0]
+        assert other.register_job(**job.hparams()) == 0
+        every = configs.rounds_all(cfg)[0]
+        for it in range(2):
+            pair.push_iteration(it)
+            pair.aggregate(every)
+        side = torch.cuda.Stream()
+        nbytes, step = pair.svc.block_export(0, 0)
+        assert step == 2
+        lane = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        assert pair.svc.block_export(0, 0, lane, nbytes, side) == (nbytes, 2)   # ordered after the aggregate
+        other.register_block(0, 0, 70001, 0, None)
+        other.block_import(0, 0, lane, nbytes, step, side)                   # same stream: after the export
+        pair.svc.unregister_block(0, 0)                                       # waits for the export
+        with pytest.raises(B.PsError):
+            pair.svc.pull(0, 0)
+        for it in range(2, 4):
+            slab = generate.grad_slab(cfg, 0, it)
+            dslab = generate.to_device(slab, "cuda")
+            host = to_np(slab)
+            for blk in job.blocks:
+                svc = other if blk.block == 0 else pair.svc
+                for w in range(job.num_workers):
+                    svc.push(0, blk.block, w, generate.shard_ptr(dslab, w, blk.job_offset))
+                    pair.ora.push(0, blk.block, w, host[w, blk.job_offset:blk.job_offset + blk.nelem])
+            # another stream than the import's, and no synchronize in between: the
+            # library itself must keep the update behind the copy
+            other.aggregate([(0, 0)], torch.cuda.Stream())
+            pair.svc.aggregate([(0, 1)])
+            pair.ora.aggregate(every)
+            torch.cuda.synchronize()
+        n = 70001
+        s0, s1, _ = other.block_state(0, 0)
+        ra, rv = pair.ora.state(0, 0)
+        assert np.array_equal(other.view(other.pull(0, 0), n).cpu().numpy(), pair.ora.pull(0, 0))
+        assert np.array_equal(other.view(s0, n).cpu().numpy(), ra)
+        if rv is not None:
+            assert np.array_equal(other.view(s1, n).cpu().numpy(), rv)
+        sq, st = other.block_stats(0, 0)
+        rsq, rst = pair.ora.block_stats(0, 0)
+        assert st == rst == 4 and abs(sq - rsq) <= 1e-5 * rsq
+        assert np.array_equal(pair.svc.view(pair.svc.pull(0, 1), 4096).cpu().numpy(), pair.ora.pull(0, 1))
+    finally:
+        pair.close()
+        other.close()
