@@ -383,6 +383,20 @@ int ps_peer_open(int device, const unsigned char* handle, void** dev_ptr_out);
 int ps_peer_close(int device, void* dev_ptr);
 const char* ps_peer_last_error(void);
 
+/* Pull from another process (paper Section 4: Pull returns the current
+ * parameters of (job, tensor)).  ps_arena_export writes the handle of a
+ * context's arena, which a worker process maps with ps_peer_open;
+ * ps_block_location says where in that arena a block lives: its parameters are
+ * the nelem floats at `offset`, its optimizer state follows in sections of
+ * `section` bytes.  The location changes when the block migrates; the contents
+ * are defined once the owner's last aggregate of the block has completed (the
+ * processes order that between themselves, as for peer buffers).  The mapping
+ * is for reading: a writer other than the owner's kernels breaks the service.
+ * Errors: BAD_ARG, NO_DEVICE, CUDA. */
+int ps_arena_export(ps_service* svc, int ctx, unsigned char* handle_out, size_t* bytes_out);
+int ps_block_location(ps_service* svc, int job, int block, int* ctx_out, size_t* offset_out,
+                      size_t* section_bytes_out);
+
 /* ---------------------------------------------------------------------------
  * Planner: which Aggregator (context) runs which aggregation task.  Host only.
  *

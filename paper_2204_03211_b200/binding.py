@@ -103,6 +103,9 @@ _SIGNATURES = {
                                  C.POINTER(C.c_ulonglong), C.c_void_p]),
     "ps_block_import": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_ulonglong, C.c_void_p]),
     "ps_unregister_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int]),
+    "ps_arena_export": (C.c_int, [C.c_void_p, C.c_int, C.c_char_p, C.POINTER(C.c_size_t)]),
+    "ps_block_location": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_size_t),
+                                   C.POINTER(C.c_size_t)]),
     "ps_peer_alloc": (C.c_int, [C.c_int, C.c_size_t, C.POINTER(C.c_void_p), C.c_char_p]),
     "ps_peer_free": (C.c_int, [C.c_int, C.c_void_p]),
     "ps_peer_open": (C.c_int, [C.c_int, C.c_char_p, C.POINTER(C.c_void_p)]),
@@ -460,6 +463,21 @@ def ps_unregister_block(svc, job: int, block: int):
     _check(load().ps_unregister_block(svc, job, block), "ps_unregister_block", svc)
 
 
+def ps_arena_export(svc, ctx: int):
+    """Returns (64-byte handle, arena bytes) of a context's arena for ps_peer_open in another process."""
+    handle, n = C.create_string_buffer(PS_PEER_HANDLE_BYTES), C.c_size_t()
+    _check(load().ps_arena_export(svc, ctx, handle, C.byref(n)), "ps_arena_export", svc)
+    return handle.raw, n.value
+
+
+def ps_block_location(svc, job: int, block: int):
+    """Returns (context, byte offset of the parameters in its arena, bytes per section)."""
+    ctx, off, sec = C.c_int(), C.c_size_t(), C.c_size_t()
+    _check(load().ps_block_location(svc, job, block, C.byref(ctx), C.byref(off), C.byref(sec)),
+           "ps_block_location", svc)
+    return ctx.value, off.value, sec.value
+
+
 def _check_peer(rc: int, where: str):
     if rc != PS_OK:
         raise PsError(rc, where, load().ps_peer_last_error().decode() if rc == PS_ERR_CUDA else "")
@@ -502,5 +520,5 @@ def _bind(name):
 
 for _n in ("register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "aggregate", "join", "pull", "pull_batch", "pull_host",
            "migrate_block", "migrate_blocks", "block_stats", "block_profile", "job_profile", "block_state", "plan", "set_option", "get_option", "arena_info",
-           "launch_info", "device_status", "block_export", "block_import", "unregister_block"):
+           "launch_info", "device_status", "block_export", "block_import", "unregister_block", "arena_export", "block_location"):
     setattr(Service, _n, _bind(_n))

@@ -1274,6 +1274,32 @@ int ps_arena_info(ps_service* s, int ctx, size_t* used_out, size_t* largest_free
   return PS_OK;
 }
 
+int ps_arena_export(ps_service* s, int ctx, unsigned char* handle_out, size_t* bytes_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (ctx < 0 || ctx >= (int)s->ctxs.size() || !handle_out) return PS_ERR_BAD_ARG;
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  PS_CUDA(s, cudaSetDevice(s->device));
+  cudaIpcMemHandle_t h;
+  static_assert(sizeof(h) == PS_PEER_HANDLE_BYTES, "handle size");
+  PS_CUDA(s, cudaIpcGetMemHandle(&h, s->ctxs[ctx].base));
+  std::memcpy(handle_out, &h, sizeof(h));
+  if (bytes_out) *bytes_out = s->ctxs[ctx].arena.capacity();
+  return PS_OK;
+}
+
+int ps_block_location(ps_service* s, int job, int block, int* ctx_out, size_t* offset_out, size_t* section_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  const int bi = find_block(s, job, block);
+  if (bi < 0) return PS_ERR_BAD_ARG;
+  const Block& b = s->blocks[bi];
+  if (ctx_out) *ctx_out = b.ctx;
+  if (offset_out) *offset_out = b.off;
+  if (section_out) *section_out = b.sec;
+  return PS_OK;
+}
+
 int ps_launch_info(ps_service* s, unsigned long long* launches, int* grid, int* block, const char** name) {
   if (!alive(s)) return PS_ERR_BAD_HANDLE;
   std::lock_guard<std::mutex> lk(s->mu);

@@ -184,6 +184,7 @@ class ShardedWorkload:
                 self.row_off[(j, w)] = size[r]
                 size[r] += row
         self.slabs = PeerSlabs(rank, world, device, size[rank], exchange)
+        self._arena_base = None
         for j, job in enumerate(cfg.jobs):
             assert self.sh.register_job(**job.hparams()) == j
             p0 = generate.init_params(cfg, j, param_device)     # the seeded generator of that device kind
@@ -198,6 +199,7 @@ class ShardedWorkload:
         import torch
         torch.cuda.synchronize(self.device)
         self.barrier()                          # nobody reads a peer's buffer any more
+        self.close_arenas()
         self.slabs.close()
         self.sh.close()
 
@@ -226,6 +228,35 @@ class ShardedWorkload:
             del slab
         torch.cuda.synchronize(dev)
         self.barrier()
+
+    def open_arenas(self, exchange):
+        """Collective: every rank exports the arenas of its service and tells where
+        its blocks live; afterwards `param_address` works for every block.  Call
+        again after a migration (locations change)."""
+        self.close_arenas()
+        nctx = self.cfg.num_contexts
+        mine = [self.sh.svc.arena_export(c)[0] for c in range(nctx)]
+        where = {k: self.sh.svc.block_location(*k)[:2] for k, r in self.sh.owner.items() if r == self.rank}
+        self._arena_base, self._where = [None] * self.world, {}
+        for r, (handles, loc) in enumerate(exchange((mine, where))):
+            self._where.update(loc)
+            if r != self.rank:
+                self._arena_base[r] = [B.ps_peer_open(self.device, h) for h in handles]
+
+    def close_arenas(self):
+        for bases in getattr(self, "_arena_base", None) or []:
+            for p in bases or []:
+                B.ps_peer_close(self.device, p)
+        self._arena_base = None
+
+    def param_address(self, job: int, block: int) -> int:
+        """Pull from anywhere: address, in this process, of the block's nelem fp32
+        parameters — in the local arena or in the owner's mapped one."""
+        r = self.sh.owner[(job, block)]
+        if r == self.rank:
+            return self.sh.pull(job, block)
+        ctx, off = self._where[(job, block)]
+        return self._arena_base[r][ctx] + off
 
     def packed_bytes(self, job: int, block: int) -> int:
         """Size of a block's packed state (parameters and optimizer state, each

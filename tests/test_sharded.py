@@ -181,6 +181,17 @@ def _gpu_rank(rank, world, port, out):
         rsq, rstep = ora.block_stats(j, blk)
         ok &= step == rstep == 3 and abs(sq - rsq) <= 1e-5 * abs(rsq) + 1e-300
         checked += 1
+    # Pull across ranks: the other rank's blocks, read in place from its mapped arena
+    wl.open_arenas(exchange)
+    pulled = 0
+    for (j, blk) in every:
+        if wl.sh.owns(j, blk):
+            continue
+        n = cfg.jobs[j].blocks[blk].nelem
+        raw = sharded.device_bytes(wl.param_address(j, blk), 4 * n, 0).cpu().numpy().view(np.float32)
+        ok &= np.array_equal(raw, ora.pull(j, blk))
+        pulled += 1
+    dist.barrier()
     gone = [k for k in every if not wl.sh.owns(*k)]
     for (j, blk) in gone[:2]:                                      # a block that left is unknown here
         try:
@@ -189,7 +200,7 @@ def _gpu_rank(rank, world, port, out):
         except B.PsError as e:
             ok &= e.status == B.PS_ERR_BAD_ARG
     with open(out % rank, "w") as f:
-        json.dump({"ok": bool(ok), "checked": checked, "remote_reads": remote_reads, "adopted": len(adopted),
+        json.dump({"ok": bool(ok), "checked": checked, "pulled": pulled, "remote_reads": remote_reads, "adopted": len(adopted),
                    "sent": sent, "status": wl.sh.svc.device_status()}, f)
     wl.close()
     dist.barrier()
@@ -203,6 +214,7 @@ def test_two_processes_on_one_device_read_each_others_shards_in_place(tmp_path):
     got = [json.load(open(out % r)) for r in range(2)]
     assert all(g["ok"] and g["status"] == 0 for g in got), got
     assert sum(g["checked"] for g in got) == 9 and min(g["checked"] for g in got) >= 2
+    assert all(g["checked"] + g["pulled"] == 9 for g in got)       # the rest was pulled from the other rank's arena
     assert all(g["remote_reads"] > 0 for g in got)                 # each rank consumed shards hosted by the other
     assert all(g["adopted"] >= 2 and g["sent"] > 0 for g in got)   # and blocks changed owner in both directions
 
