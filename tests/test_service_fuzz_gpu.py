@@ -1,7 +1,8 @@
 """Seeded random operation sequences against the service and the oracle side by
 side: registrations, dense and row-sparse pushes in any order, aggregates of
-random ready subsets on random streams, migrations, and calls that must fail
-without changing anything.  After every aggregate the touched blocks are
+random ready subsets on random streams, migrations, blocks that leave the
+service (their ids are not reused here: the oracle has no such call), and calls
+that must fail without changing anything.  After every aggregate the touched blocks are
 compared bit for bit."""
 import numpy as np
 import pytest
@@ -33,6 +34,7 @@ def test_random_operation_sequences(seed):
     ora = A.OracleAggregator(nctx)
     streams = [None, torch.cuda.Stream(), torch.cuda.Stream()]
     jobs, blocks = [], {}            # blocks[(j, b)] = dict(n, rows, pushed=set)
+    next_id = {}                     # per job: ids handed out so far
     keep = []
     aggregated = 0
     try:
@@ -48,7 +50,8 @@ def test_random_operation_sequences(seed):
                 jobs.append(kw)
             elif op < 0.12 or not blocks:
                 j = int(rng.integers(len(jobs)))
-                b = len([k for k in blocks if k[0] == j])
+                b = next_id.get(j, 0)
+                next_id[j] = b + 1
                 rows = int(rng.integers(1, 300))
                 n = rows * ROW if rng.random() < 0.6 else int(rng.integers(1, 20000))
                 ctx = int(rng.integers(nctx))
@@ -84,6 +87,16 @@ def test_random_operation_sequences(seed):
                     svc.push(j, b, w, d)
                     ora.push(j, b, w, as_np(g))
                 st["pushed"].add(w)
+            elif op < 0.635 and len(blocks) > 3:
+                # a block leaves the service (e.g. it moved to another Aggregator): whatever is
+                # enqueued for it completes first, its arena range returns, its id is unknown afterwards
+                (j, b), st = list(blocks.items())[int(rng.integers(len(blocks)))]
+                used = sum(svc.arena_info(c)[0] for c in range(nctx))
+                svc.unregister_block(j, b)
+                del blocks[(j, b)]
+                assert sum(svc.arena_info(c)[0] for c in range(nctx)) < used
+                assert _status(svc.pull, j, b) == B.PS_ERR_BAD_ARG
+                assert _status(svc.unregister_block, j, b) == B.PS_ERR_BAD_ARG
             elif op < 0.72:
                 (j, b), st = list(blocks.items())[int(rng.integers(len(blocks)))]
                 dst = int(rng.integers(nctx))
