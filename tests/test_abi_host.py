@@ -198,3 +198,21 @@ def test_arena_accounting_and_exhaustion():
     assert s.arena_info(0)[0] == 3 * 4096            # failed registration left nothing behind
     s.register_block(j, 1, 80_000)
     assert s.arena_info(0)[0] == 3 * 4096 + 3 * 320_000
+
+
+def test_plain_c99_client_compiles_against_the_header_and_runs(tmp_path):
+    """The boundary is C: a C99 program built with gcc -pedantic against
+    include/ps_b200.h links the library and exercises registration, push
+    bookkeeping, packing and the error codes on a planning-only service."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no gcc")
+    exe = str(tmp_path / "abi_client")
+    libdir = os.path.dirname(B.LIB_PATH)
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                    "-o", exe, os.path.join(ROOT, "tests", "c", "abi_client.c"), "-L", libdir, "-lps_b200",
+                    "-Wl,-rpath," + libdir], check=True, capture_output=True, text=True)
+    r = subprocess.run([exe], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+    assert "abi_client: ok" in r.stdout
