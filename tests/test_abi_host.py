@@ -216,3 +216,25 @@ def test_plain_c99_client_compiles_against_the_header_and_runs(tmp_path):
     r = subprocess.run([exe], capture_output=True, text=True)
     assert r.returncode == 0, r.stderr
     assert "abi_client: ok" in r.stdout
+
+
+@pytest.mark.gpu
+def test_plain_c99_client_computes_on_the_gpu(tmp_path):
+    """The same boundary with a device: a C99 program (CUDA runtime for memory,
+    no Python, no torch) aggregates W identical shards twice and checks the
+    hand-worked momentum recurrence exactly."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no gcc")
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    exe = str(tmp_path / "abi_gpu_client")
+    libdir = os.path.dirname(B.LIB_PATH)
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                    "-isystem", os.path.join(cuda, "include"), "-o", exe, os.path.join(ROOT, "tests", "c", "abi_gpu_client.c"),
+                    "-L", libdir, "-lps_b200", "-L", os.path.join(cuda, "lib64"), "-lcudart",
+                    "-Wl,-rpath," + libdir, "-Wl,-rpath," + os.path.join(cuda, "lib64")],
+                   check=True, capture_output=True, text=True)
+    r = subprocess.run([exe], capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr
+    assert "abi_gpu_client: ok" in r.stdout
