@@ -232,8 +232,11 @@ int grow_dev(ps_service* s, T** buf, size_t* cap, size_t need, bool zero_new) {
   if (zero_new) PS_CUDA(s, cudaMemset(nbuf, 0, ncap * sizeof(T)));
   if (*buf) {
     PS_CUDA(s, cudaMemcpy(nbuf, *buf, *cap * sizeof(T), cudaMemcpyDeviceToDevice));
-    PS_CUDA(s, cudaFree(*buf));
   }
+  // device memsets and device-to-device copies may return before they have run, and
+  // the service's streams do not synchronize with the default stream
+  PS_CUDA(s, cudaStreamSynchronize(cudaStreamLegacy));
+  if (*buf) PS_CUDA(s, cudaFree(*buf));
   *buf = nbuf;
   *cap = ncap;
   return PS_OK;
@@ -446,6 +449,7 @@ int acquire_slot(ps_service* s, size_t table_bytes, size_t nchunks, Slot** out) 
   if (!sl.mut) {
     PS_CUDA(s, cudaMalloc(&sl.mut, kInlineMaxTasks * sizeof(PsTaskMut)));
     PS_CUDA(s, cudaMemset(sl.mut, 0, kInlineMaxTasks * sizeof(PsTaskMut)));   // kept all-zero by the kernel
+    PS_CUDA(s, cudaStreamSynchronize(cudaStreamLegacy));                      // before a service stream uses it
   }
   sl.gen = s->gen;
   *out = &sl;
@@ -518,6 +522,7 @@ int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes
       e = cudaStreamCreateWithFlags(&s->work_streams[i], cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaMalloc(&s->status_dev, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(s->status_dev, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaStreamSynchronize(cudaStreamLegacy);
     for (int c = 0; e == cudaSuccess && c < num_contexts; ++c) {
       void* base = nullptr;
       e = cudaMalloc(&base, s->ctxs[c].arena.capacity() ? s->ctxs[c].arena.capacity() : Arena::kAlign);
