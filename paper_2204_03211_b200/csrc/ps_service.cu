@@ -594,6 +594,7 @@ int ps_register_job(ps_service* s, const ps_job_desc* d, int* job_out) {
     jd.omb2 = 1.0f - d->beta2;
     jd.eps = d->eps; jd.gs = d->grad_scale;
     PS_CUDA(s, cudaMemcpy(s->jobs_dev + id, &jd, sizeof jd, cudaMemcpyHostToDevice));
+    PS_CUDA(s, cudaStreamSynchronize(cudaStreamLegacy));   // a small pageable copy may still be in flight on return
   }
   Job j;
   j.d = *d;
