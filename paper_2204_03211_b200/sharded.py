@@ -67,12 +67,16 @@ class PeerSlabs:
                 self.base[r] = B.ps_peer_open(device, h)
                 self._opened.append(self.base[r])
 
-    def close(self):
+    def close(self, barrier=None):
         """Unmaps the peers' buffers and frees this rank's own.  Call it on every
-        rank only after all ranks have finished using the buffers."""
+        rank only after all ranks have finished using the buffers.  With
+        `barrier` (a callable every rank calls) no rank frees its buffer before
+        every rank has unmapped it."""
         for p in self._opened:
             B.ps_peer_close(self.device, p)
         self._opened = []
+        if barrier is not None:
+            barrier()
         if self.own:
             B.ps_peer_free(self.device, self.own)
             self.own = 0
@@ -200,7 +204,8 @@ class ShardedWorkload:
         torch.cuda.synchronize(self.device)
         self.barrier()                          # nobody reads a peer's buffer any more
         self.close_arenas()
-        self.slabs.close()
+        self.barrier()                          # every mapping of an arena is gone before its service goes
+        self.slabs.close(self.barrier)
         self.sh.close()
 
     def shard_address(self, job: int, block: int, worker: int) -> int:
@@ -310,7 +315,7 @@ class ShardedWorkload:
             self.sh.svc.unregister_block(j, b)
         for (j, b, r) in moves:
             self.sh.owner[(j, b)] = r
-        lane.close()
+        lane.close(self.barrier)
         self._args.clear()
         self.owned_params = sum(self.cfg.jobs[j].blocks[b].nelem for (j, b), r in self.sh.owner.items() if r == self.rank)
         self.owned_bytes = sum(self.cfg.jobs[j].bytes_per_elem() * self.cfg.jobs[j].blocks[b].nelem
