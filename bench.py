@@ -522,7 +522,8 @@ def main():
     if rank == 0:
         sampler.start()
     l0 = wl.svc.launch_info()["launches"]
-    ms, launches, host_ms = timed(lambda k, s: wl.step(args.warmup + k, s), args.steps, stream, dist_on, device)
+    red_dev = device if args.dist_backend == "nccl" else None      # where the max over ranks is reduced
+    ms, launches, host_ms = timed(lambda k, s: wl.step(args.warmup + k, s), args.steps, stream, dist_on, red_dev)
     clocks = sampler.stop() if rank == 0 else {}
     info = wl.svc.launch_info()
     assert info["launches"] - l0 == launches
@@ -540,7 +541,7 @@ def main():
         wl.prepare_host(int(args.host_pool_gb * (1 << 30)))
         wl.step_host(0, stream)         # warm-up: allocates the staging buffers
         torch.cuda.synchronize(device)
-        ems, _, _ = timed(wl.step_host, args.e2e_steps, stream, dist_on, device)
+        ems, _, _ = timed(wl.step_host, args.e2e_steps, stream, dist_on, red_dev)
         e2e = {"value": whole_job_value(wl.params_per_step, world, args.e2e_steps, ems), "unit": UNIT,
                "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "steps": args.e2e_steps,
                "ms_per_step": ems / args.e2e_steps,

@@ -323,3 +323,24 @@ def test_block_moves_between_two_services_and_training_continues_bit_for_bit(opt
     finally:
         pair.close()
         other.close()
+
+
+@pytest.mark.gpu
+def test_bench_replica_arm_two_ranks_on_one_device():
+    """The default arm of bench.py for more than one rank (independent replicas,
+    max over ranks, whole-job units), launched the way a multi-GPU run launches
+    it; here both ranks share the one device and meet over gloo."""
+    import subprocess
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
+           "127.0.0.1", "--master-port", str(_free_port()), os.path.join(ROOT, "bench.py"), "--gpus", "2",
+           "--dist-backend", "gloo", "--workload", "C1", "--steps", "20", "--warmup", "3", "--e2e-steps", "1"]
+    r = subprocess.run(cmd, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                         # rank 0 alone prints
+    line = json.loads(lines[0])
+    cfg = configs.c1()
+    assert line["n_gpus"] == 2 and line["scaling"] == "weak" and line["steps"] == 20
+    assert abs(line["value"] - 2 * cfg.num_params / (line["ms_per_step"] * 1e-3)) <= 1e-6 * line["value"]
+    assert line["gpu_launches"] == 20 and line["cpu_baseline"] is None
+    assert line["e2e"]["h2d_bytes_per_step"] == 4 * 4 * cfg.num_params
