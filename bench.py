@@ -230,6 +230,10 @@ class Workload:
         self.pull_done = torch.cuda.Event()
         self.h2d = total
         self.d2h = self.cfg.num_params * 4
+        self._out_off, acc = {}, 0
+        for j, job in enumerate(self.cfg.jobs):
+            self._out_off[j] = acc
+            acc += job.num_params
 
     def step_host(self, k: int, stream) -> int:
         svc, cfg = self.svc, self.cfg
@@ -258,6 +262,45 @@ class Workload:
                 svc.pull_host(j, b, out_ptr + 4 * (out_off[j] + cfg.jobs[j].blocks[b].job_offset), self.pull_stream)
         self.pull_done.record(self.pull_stream)
         stream.wait_event(self.pull_done)           # the step ends when its last result is on the host
+        if self.overlap:
+            svc.join(stream)
+        return len(rounds)
+
+
+    def step_host_mapped(self, k: int, stream) -> int:
+        """End to end without staging copies: pinned host memory is addressable
+        from the device, so the pinned shards are pushed as they are and the
+        aggregation kernel reads them over PCIe in place; parameters return to
+        the host as in step_host."""
+        svc, cfg = self.svc, self.cfg
+        rounds = self.schedules[k % len(self.schedules)]
+        if not hasattr(self, "_mapped_args"):
+            self._mapped_args = {}
+        out_ptr = self.out.data_ptr()
+        for i, r in enumerate(rounds):
+            key = (k % len(self.schedules), i)
+            if key not in self._mapped_args:
+                # where each (block, worker) shard of this round sits in the pinned pool
+                jobs, blocks, workers, ptrs = [], [], [], []
+                cursor = 0
+                for (j, b) in r["ready"]:
+                    job = cfg.jobs[j]
+                    nbytes = job.blocks[b].nelem * (2 if job.grad_dtype == configs.BF16 else 4)
+                    for w in range(job.num_workers):
+                        if cursor + nbytes > self.pool_bytes:
+                            cursor = 0
+                        jobs.append(j); blocks.append(b); workers.append(w)
+                        ptrs.append(self.pool.data_ptr() + cursor)
+                        cursor += (nbytes + 255) // 256 * 256
+                self._mapped_args[key] = (np.array(jobs, np.int32), np.array(blocks, np.int32),
+                                          np.array(workers, np.int32), np.array(ptrs, np.uint64))
+            svc.push_batch(*self._mapped_args[key])
+            svc.aggregate(r["tasks"], stream)
+            for (j, b) in r["ready"]:
+                svc.pull_host(j, b, out_ptr + 4 * (self._out_off[j] + cfg.jobs[j].blocks[b].job_offset),
+                              self.pull_stream)
+        self.pull_done.record(self.pull_stream)
+        stream.wait_event(self.pull_done)
         if self.overlap:
             svc.join(stream)
         return len(rounds)
@@ -428,6 +471,10 @@ def main():
     ap.add_argument("--workload", default="C4", choices=sorted(configs.CONFIGS))
     ap.add_argument("--ticks", type=int, default=16, help="rounds per iteration window of the arrival schedule")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-mode", default="mapped", choices=["staged", "mapped"],
+                    help="staged: only the e2e leg whose shards ps_push_host copies into device staging; mapped: "
+                         "also a second leg (e2e_mapped) whose pinned shards are pushed as they are and read by "
+                         "the kernel over PCIe")
     ap.add_argument("--host-pool-gb", type=float, default=8.0)
     ap.add_argument("--jobs", default="", help="comma-separated subset of the workload's jobs (profiling a small case)")
     ap.add_argument("--max-blocks", type=int, default=0, help="keep only the first N blocks of every job")
@@ -536,16 +583,23 @@ def main():
     if NCU_TRAFFIC["kernel_sha"] == sha and NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"]:
         traffic = per_launch_bytes * NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"]
 
-    e2e = None
+    e2e = e2e_mapped = None
     if not args.no_e2e:
         wl.prepare_host(int(args.host_pool_gb * (1 << 30)))
-        wl.step_host(0, stream)         # warm-up: allocates the staging buffers
-        torch.cuda.synchronize(device)
-        ems, _, _ = timed(wl.step_host, args.e2e_steps, stream, dist_on, red_dev)
-        e2e = {"value": whole_job_value(wl.params_per_step, world, args.e2e_steps, ems), "unit": UNIT,
-               "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "steps": args.e2e_steps,
-               "ms_per_step": ems / args.e2e_steps,
-               "host_pool_bytes": wl.pool_bytes}
+        def host_leg(host_step, mode):
+            host_step(0, stream)        # warm-up (staged: allocates the staging buffers)
+            torch.cuda.synchronize(device)
+            ems, _, _ = timed(host_step, args.e2e_steps, stream, dist_on, red_dev)
+            return {"value": whole_job_value(wl.params_per_step, world, args.e2e_steps, ems), "unit": UNIT,
+                    "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "steps": args.e2e_steps,
+                    "ms_per_step": ems / args.e2e_steps, "mode": mode, "host_pool_bytes": wl.pool_bytes}
+
+        # staged: ps_push_host copies every shard from pinned memory into device staging, then the kernel
+        # reads the staging; mapped: the pinned shards themselves are pushed (ps_push) and the kernel
+        # reads them over PCIe in place.  Same bytes cross the link every step in both.
+        e2e = host_leg(wl.step_host, "staged: ps_push_host copies, then aggregate")
+        if args.e2e_mode == "mapped":
+            e2e_mapped = host_leg(wl.step_host_mapped, "mapped: ps_push of pinned host pointers, the kernel reads over PCIe")
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -566,7 +620,7 @@ def main():
                          "bytes_per_launch": per_launch_bytes, "kernel_sha": sha,
                          "note": "duration = event time of the whole timed region / launches "
                                  "(launches of a step may overlap; table uploads included)"},
-            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+            "cpu_baseline": cpu, "e2e": e2e, "e2e_mapped": e2e_mapped, "gpu_launches": launches,
             "launch": {"grid": info["grid"], "block": info["block"]},
             "host_ms_per_step": host_ms / args.steps, "clocks": clocks,
         }

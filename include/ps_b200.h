@@ -132,7 +132,10 @@ int ps_register_block(ps_service* svc, int job, int block, size_t nelem, int ctx
  * contiguous values of the job's grad_dtype; it must stay valid and unmodified
  * until the ps_aggregate that consumes it has completed on its stream.  The
  * task is ready once all W workers have pushed.  16-byte aligned pointers take
- * the vector path, others a scalar path with identical results.
+ * the vector path, others a scalar path with identical results.  Any address
+ * the service's GPU can load from will do: its own memory, a mapped peer buffer
+ * (ps_peer_open), or page-locked host memory (cudaHostAlloc / cudaHostRegister
+ * under unified addressing), which the kernel then reads over PCIe in place.
  * Errors: BAD_ARG, DUPLICATE (this worker already pushed this iteration; the
  * paper has one request per task per iteration), ALIGN. */
 int ps_push(ps_service* svc, int job, int block, int worker, const void* grad_dev_ptr);

@@ -234,3 +234,30 @@ def test_sqnorm_all_ones_and_host_push_pull():
         assert torch.equal(out, p0 - 0.5 * 2.0)
     finally:
         pair.close()
+
+
+@pytest.mark.parametrize("opt,dt", [(configs.SGD, configs.F32), (configs.ADAM, configs.BF16)])
+def test_pinned_host_shards_are_read_in_place(opt, dt):
+    """Pinned host memory is addressable from the device: ps_push takes the
+    pinned pointer and the kernel reads the shard over PCIe, no staging copy."""
+    cfg = tiny_config([70001, 4096, 33], 3, opt=opt, grad_dtype=dt)
+    pair = Pair(cfg)
+    try:
+        job = cfg.jobs[0]
+        every = configs.rounds_all(cfg)[0]
+        for it in range(2):
+            slab = generate.grad_slab(cfg, 0, it)
+            pinned = generate.empty_slab(slab.shape[0], slab.shape[1], slab.dtype, "cpu")
+            base = pinned._base.pin_memory()                     # same padded row layout, page-locked
+            pinned = base[:, :slab.shape[1]]
+            pinned.copy_(slab)
+            host = to_np(slab)
+            for b in job.blocks:
+                for w in range(job.num_workers):
+                    pair.svc.push(0, b.block, w, generate.shard_ptr(pinned, w, b.job_offset))
+                    pair.ora.push(0, b.block, w, host[w, b.job_offset:b.job_offset + b.nelem])
+            pair.aggregate(every)
+            torch.cuda.synchronize()                             # the pinned buffer is released after this
+        pair.compare()
+    finally:
+        pair.close()
