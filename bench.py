@@ -180,28 +180,32 @@ class Workload:
                 r["c_push"] = (len(r["jobs"]), r["jobs"].ctypes.data, r["blocks"].ctypes.data,
                                r["workers"].ctypes.data, r["ptrs"].ctypes.data)
                 r["c_pulled"] = r["pulled"].ctypes.data
+                r["c_round"] = r["c_push"] + (r["tasks"], r["n"])
                 if r["rows"] is not None:
                     r["c_rows"] = (len(r["rows"][0]),) + tuple(a.ctypes.data for a in r["rows"])
             self.schedules.append(rounds)
         self.lib = B.load()
         self.overlap = False
+        # the gradient slabs are written once, before any timed region: every push is of a
+        # buffer that is already complete in memory
+        self.round_flags = B.PS_ROUND_INPUTS_COMPLETE
         self.params_per_step = cfg.num_params
         self.bytes_per_step = cfg.bytes_per_round() - self.sparse_saved
 
     def step(self, k: int, stream) -> int:
         """Push, aggregate, pull — device-resident gradients.  Returns launches."""
         # The C entry points are called with arguments marshalled once, outside
-        # the timed region (array addresses as integers): three C-ABI calls per round.
+        # the timed region (array addresses as integers): one C-ABI call per round
+        # (ps_round = push, aggregate, pull), plus one for row-sparse pushes if any.
         lib, h, sp = self.lib, self.svc.handle, int(stream.cuda_stream)
         rounds = self.schedules[k % len(self.schedules)]
+        flags = self.round_flags
         for r in rounds:
-            rc = lib.ps_push_batch(h, *r["c_push"])
-            if rc == 0 and r["rows"] is not None:
+            rc = 0
+            if r["rows"] is not None:
                 rc = lib.ps_push_rows_batch(h, *r["c_rows"])
             if rc == 0:
-                rc = lib.ps_aggregate(h, r["tasks"], r["n"], sp)
-            if rc == 0:
-                rc = lib.ps_pull_batch(h, r["tasks"], r["n"], r["c_pulled"])
+                rc = lib.ps_round(h, *r["c_round"], flags, sp, r["c_pulled"])
             if rc:
                 raise self.B.PsError(rc, "bench step")
         if self.overlap:
@@ -491,6 +495,7 @@ def main():
                          "shards are read in place from the worker ranks' exported buffers) instead of N replicas")
     ap.add_argument("--dist-backend", default="nccl", choices=["nccl", "gloo"],
                     help="process-group backend for the barriers and the max over ranks")
+    ap.add_argument("--no-pdl", action="store_true", help="PS_OPT_PDL = 0: plain launches for small rounds")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -558,6 +563,7 @@ def main():
             wl.sparse_saved / 1e9)
     wl.svc.set_option(wl.B.PS_OPT_CHUNK_ELEMS, args.chunk_elems)
     wl.svc.set_option(wl.B.PS_OPT_KERNEL, args.kernel)
+    wl.svc.set_option(wl.B.PS_OPT_PDL, int(not args.no_pdl))
     wl.overlap = not args.in_stream
     wl.svc.set_option(wl.B.PS_OPT_OVERLAP, int(wl.overlap))
     config["launch_mode"] = "overlapped, one ps_join per step" if wl.overlap else "in-stream"

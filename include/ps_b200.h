@@ -87,10 +87,19 @@ enum {
                               gradient buffers or reads results on its own streams; ps_pull_host,
                               ps_block_stats, ps_block_profile, ps_migrate_block and ps_push_host
                               order themselves after the block's last launch in either mode.
+                              A launch that must follow an unfinished one (a block aggregated again)
+                              goes to that launch's stream; completion is learnt from a word each
+                              kernel stores to page-locked host memory, so a launch costs no event
+                              unless another stream has to wait for it.
                               Default 0: every launch is enqueued on `stream` itself. */
   PS_OPT_INLINE_TABLE = 7, /* 1 (default): a launch whose task table fits 3968 bytes (a round of a few
                               tensors) and has few chunks passes the table as a kernel parameter, one
                               CTA per chunk: no upload.  0: always upload the table.  Same results. */
+  PS_OPT_PDL = 8,          /* 1 (default): such small launches carry the programmatic-stream-serialization
+                              launch attribute: the kernel's prologue (task lookup in its parameters)
+                              overlaps the tail of the previous launch of the same stream, and the
+                              kernel waits for that launch to complete before it touches any data.
+                              0: plain launches.  Same results. */
   PS_OPT_PROFILE = 5,      /* 1: aggregates record per-task device time (see ps_block_profile);
                               costs a few atomics per chunk; direct-load kernel only; default 0 */
   PS_OPT_KERNEL = 4        /* kernel variant: 0 = automatic (direct loads), 1 = direct loads,
@@ -152,8 +161,12 @@ int ps_push(ps_service* svc, int job, int block, int worker, const void* grad_de
  * row_len * element size a multiple of 16 bytes; `values` 16-byte aligned (else
  * PS_ERR_ALIGN); W <= 32.  n_rows may be 0 (both pointers still non-NULL).  A
  * block may receive dense pushes from some workers and row-sparse ones from
- * others, all with the same row_len within an iteration.  Launches that carry
- * such tasks always use the direct-load kernel.
+ * others, all with the same row_len within an iteration; the dense shards of
+ * such a block are streamed row by row with 128-bit loads as well, so they must
+ * be 16-byte aligned too: whichever push comes second (the row-sparse one after
+ * an unaligned dense one, or the unaligned dense one after a row-sparse one) is
+ * rejected with PS_ERR_ALIGN.  Launches that carry such tasks always use the
+ * direct-load kernel.
  * Errors: BAD_ARG, ALIGN, DUPLICATE. */
 int ps_push_rows(ps_service* svc, int job, int block, int worker, const int* row_ids_dev, int n_rows,
                  int row_len, const void* values_dev);
@@ -191,6 +204,27 @@ int ps_aggregate(ps_service* svc, const ps_task* ready, int n_ready, void* strea
 /* Makes `stream` wait for every ps_aggregate launch enqueued so far that it has
  * not joined yet (needed only with PS_OPT_OVERLAP; otherwise a no-op). */
 int ps_join(ps_service* svc, void* stream);
+
+/* One round of the service in ONE call — what an Aggregator does when the last
+ * worker's gradients of some tensors have arrived (paper Figure 1 and Section 2.1:
+ * tensors become ready one layer after another during the backward pass, so a
+ * round is often a few small tensors and its cost is the cost of the calls):
+ * the n_push pushes of ps_push_batch, then ps_aggregate(ready, n_ready, stream),
+ * then, if params_dev_ptrs_out is not NULL, the n_ready parameter pointers of
+ * ps_pull_batch (in the order of `ready`).  All-or-nothing: when the aggregate is
+ * rejected the pushes of this call are taken back.
+ * flags: PS_ROUND_INPUTS_COMPLETE — every gradient buffer pushed for the listed
+ * tasks is already complete in memory when the call is made (it arrived over the
+ * network or a peer link and the host was told; nothing still enqueued on
+ * `stream` writes it).  With PS_OPT_OVERLAP the launch then does not wait for
+ * `stream` at all, and a round costs the host one kernel launch.  Without the
+ * flag the launch is ordered after the work enqueued on `stream`, as for
+ * ps_aggregate.
+ * Errors: those of ps_push_batch and ps_aggregate; BAD_ARG for unknown flags. */
+#define PS_ROUND_INPUTS_COMPLETE 1u
+int ps_round(ps_service* svc, int n_push, const int* jobs, const int* blocks, const int* workers,
+             const void* const* grad_dev_ptrs, const ps_task* ready, int n_ready, unsigned int flags,
+             void* stream, const float** params_dev_ptrs_out);
 
 /* Pull (paper Section 4): *params_dev_ptr_out receives a device pointer to the
  * block's nelem fp32 parameters.  Borrowed; stable until the block is migrated
@@ -274,10 +308,24 @@ int ps_get_option(ps_service* svc, int option, long long* value_out);
 /* Bytes in use / largest free range of a context's arena. */
 int ps_arena_info(ps_service* svc, int ctx, size_t* used_out, size_t* largest_free_out);
 
+/* Size of the registry: registered jobs, registered blocks, and entries of the
+ * block table (registered blocks plus entries that ps_unregister_block released
+ * and a later ps_register_block will use again — the table does not grow while
+ * blocks come and go). */
+int ps_registry_info(ps_service* svc, size_t* jobs_out, size_t* blocks_out, size_t* block_entries_out);
+
 /* Number of aggregation kernels launched so far and the grid/block size and
  * variant name of the last one (for launch accounting in benchmarks). */
 int ps_launch_info(ps_service* svc, unsigned long long* launches_out, int* grid_out, int* block_out,
                    const char** kernel_name_out);
+
+/* Launch accounting per kernel variant (0 = persistent direct-load kernel,
+ * 1 = small-launch kernel with the table in its parameters, 2 = bulk-copy ring):
+ * launches so far, the algorithmic bytes they covered (W shards read, parameters
+ * and state read and written, dense semantics) and the kernel's name.
+ * Errors: BAD_ARG (variant out of range). */
+int ps_launch_stats(ps_service* svc, int variant, unsigned long long* launches_out,
+                    unsigned long long* algorithmic_bytes_out, const char** kernel_name_out);
 
 /* Waits for the device and reports the kernels' status word: 0 = no fault;
  * non-zero = a bounded wait inside a kernel expired (the launch returned early

@@ -27,6 +27,8 @@ PS_PEER_HANDLE_BYTES = 64
 PS_OPT_CHUNK_ELEMS, PS_OPT_CTAS_PER_SM, PS_OPT_SORT_TASKS, PS_OPT_KERNEL, PS_OPT_PROFILE = 1, 2, 3, 4, 5
 PS_OPT_OVERLAP = 6
 PS_OPT_INLINE_TABLE = 7
+PS_OPT_PDL = 8
+PS_ROUND_INPUTS_COMPLETE = 1
 
 
 class ps_job_desc(C.Structure):
@@ -65,6 +67,10 @@ _SIGNATURES = {
     "ps_push_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
     "ps_aggregate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "ps_join": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "ps_round": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                           C.c_uint, C.c_void_p, C.c_void_p]),
+    "ps_launch_stats": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_ulonglong), C.POINTER(C.c_ulonglong),
+                                  C.POINTER(C.c_char_p)]),
     "ps_pull": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p)]),
     "ps_pull_batch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "ps_pull_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
@@ -80,6 +86,7 @@ _SIGNATURES = {
     "ps_set_option": (C.c_int, [C.c_void_p, C.c_int, C.c_longlong]),
     "ps_get_option": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_longlong)]),
     "ps_arena_info": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "ps_registry_info": (C.c_int, [C.c_void_p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
     "ps_launch_info": (C.c_int, [C.c_void_p, C.POINTER(C.c_ulonglong), C.POINTER(C.c_int), C.POINTER(C.c_int),
                                  C.POINTER(C.c_char_p)]),
     "ps_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int)]),
@@ -237,6 +244,28 @@ def ps_join(svc, stream=None):
     _check(load().ps_join(svc, _stream_ptr(stream)), "ps_join", svc)
 
 
+def ps_round(svc, jobs, blocks, workers, ptrs, ready, flags: int = 0, stream=None, out=None):
+    """ps_push_batch + ps_aggregate + ps_pull_batch in one call.  jobs/blocks/
+    workers: int32 numpy arrays, ptrs: uint64 numpy array (all may be None for
+    no pushes); ready: ps_task array or list of (job, block); out: optional
+    uint64 numpy array that receives the parameter pointers."""
+    tasks = ready if isinstance(ready, C.Array) else make_tasks(list(ready))
+    n = 0 if jobs is None else len(jobs)
+    _check(load().ps_round(svc, n, _ptr(jobs), _ptr(blocks), _ptr(workers), _ptr(ptrs), tasks, len(tasks), flags,
+                           _stream_ptr(stream), _ptr(out)), "ps_round", svc)
+    return out
+
+
+def ps_launch_stats(svc):
+    """[{kernel, launches, bytes}] per kernel variant."""
+    res = []
+    for v in range(3):
+        n, b, name = C.c_ulonglong(), C.c_ulonglong(), C.c_char_p()
+        _check(load().ps_launch_stats(svc, v, C.byref(n), C.byref(b), C.byref(name)), "ps_launch_stats", svc)
+        res.append(dict(kernel=(name.value or b"").decode(), launches=n.value, bytes=b.value))
+    return res
+
+
 def ps_pull(svc, job: int, block: int) -> int:
     out = C.c_void_p()
     _check(load().ps_pull(svc, job, block, C.byref(out)), "ps_pull", svc)
@@ -315,6 +344,12 @@ def ps_arena_info(svc, ctx: int):
     return used.value, free.value
 
 
+def ps_registry_info(svc):
+    j, b, e = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    _check(load().ps_registry_info(svc, C.byref(j), C.byref(b), C.byref(e)), "ps_registry_info", svc)
+    return dict(jobs=j.value, blocks=b.value, block_entries=e.value)
+
+
 def ps_launch_info(svc):
     n, g, b, name = C.c_ulonglong(), C.c_int(), C.c_int(), C.c_char_p()
     _check(load().ps_launch_info(svc, C.byref(n), C.byref(g), C.byref(b), C.byref(name)), "ps_launch_info", svc)
@@ -326,6 +361,8 @@ def ps_aggregate_block_noalloc(job_desc: ps_job_desc, step: int, nelem: int, par
     """One block through the entry point that allocates nothing (see the
     header).  params/state0/state1/sqnorm_out: device tensors or addresses;
     shards: list of W device tensors or addresses."""
+    if len(shards) != job_desc.num_workers:
+        raise ValueError("%d shards for a job of %d workers" % (len(shards), job_desc.num_workers))
     arr = (C.c_void_p * len(shards))(*[_ptr(g) for g in shards])
     _check(load().ps_aggregate_block_noalloc(C.byref(job_desc), step, nelem, _ptr(params), _ptr(state0),
                                              _ptr(state1), arr, _ptr(sqnorm_out), _stream_ptr(stream)),
@@ -518,7 +555,7 @@ def _bind(name):
     return method
 
 
-for _n in ("register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "aggregate", "join", "pull", "pull_batch", "pull_host",
+for _n in ("round", "launch_stats", "registry_info", "register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "aggregate", "join", "pull", "pull_batch", "pull_host",
            "migrate_block", "migrate_blocks", "block_stats", "block_profile", "job_profile", "block_state", "plan", "set_option", "get_option", "arena_info",
            "launch_info", "device_status", "block_export", "block_import", "unregister_block", "arena_export", "block_location"):
     setattr(Service, _n, _bind(_n))

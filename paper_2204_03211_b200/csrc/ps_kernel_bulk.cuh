@@ -318,8 +318,7 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
       // at a CTA barrier, each publishes its own partial
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) sq += __shfl_down_sync(0xffffffffu, sq, o);
-      if (lane == 0)
-        publish_part(tasks, m.task, m.chunk * kBulkConsumerWarps + warp, kBulkConsumerWarps, sq, stats, partials);
+      publish_part(tasks, m.task, m.chunk * kBulkConsumerWarps + warp, kBulkConsumerWarps, sq, stats, partials, lane);
       sq = 0.0;
     }
   }

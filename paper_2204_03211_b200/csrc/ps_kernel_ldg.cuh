@@ -13,7 +13,8 @@ constexpr int kThreads = 256;          // threads per CTA
 
 __global__ void __launch_bounds__(kThreads, 4)
 ps_aggregate_ldg_kernel(unsigned char* __restrict__ table, const PsJobDev* __restrict__ jobs,
-                        PsStat* __restrict__ stats, double* __restrict__ partials) {
+                        PsStat* __restrict__ stats, double* __restrict__ partials,
+                        unsigned long long* done_word, unsigned long long seq) {
   PsTableHdr* hdr = reinterpret_cast<PsTableHdr*>(table);
   PsTaskDev* tasks = reinterpret_cast<PsTaskDev*>(table + hdr->tasks_off);
   const unsigned int* starts = reinterpret_cast<const unsigned int*>(table + hdr->starts_off);
@@ -62,15 +63,19 @@ ps_aggregate_ldg_kernel(unsigned char* __restrict__ table, const PsJobDev* __res
     for (int o = 16; o > 0; o >>= 1) sq += __shfl_down_sync(0xffffffffu, sq, o);
     if (lane == 0) s_red[warp] = sq;
     __syncthreads();
-    if (tid == 0) {
-      double s = s_red[0];
+    if (warp == 0) {
+      double s = 0.0;
+      if (lane == 0) {
+        s = s_red[0];
 #pragma unroll
-      for (int k = 1; k < kThreads / 32; ++k) s += s_red[k];
-      if (profile) profile_chunk(tasks + t, t_begin, global_ns());
-      publish_part(tasks, t, idx, 1u, s, stats, partials);
+        for (int k = 1; k < kThreads / 32; ++k) s += s_red[k];
+        if (profile) profile_chunk(tasks + t, t_begin, global_ns());
+      }
+      publish_part(tasks, t, idx, 1u, s, stats, partials, lane);
     }
     buf ^= 1;
   }
+  signal_exit(&hdr->exited, done_word, seq);
 }
 
 }  // namespace psb

@@ -274,6 +274,34 @@ __device__ __forceinline__ Hp load_hp(const PsJobDev* J, const PsTaskDev* T) {
 }
 
 // One chunk read with ordinary loads; dispatches on (optimizer, gradient type).
+struct JobView {                       // what a chunk body needs from its job, loaded once
+  Hp h;
+  int W, kind;                         // kind = (optimizer << 1) | gradient type
+};
+
+__device__ __forceinline__ JobView load_job(const PsJobDev* J, const PsTaskDev* T) {
+  JobView v;
+  v.h = load_hp(J, T);
+  v.W = J->W;
+  v.kind = (J->opt << 1) | J->grad_dtype;
+  return v;
+}
+
+template <int NT>
+__device__ __forceinline__ void run_chunk_view(unsigned int tid, const JobView& v, const PsTaskDev* T,
+                                               const void* const* shards, size_t begin, unsigned int count,
+                                               double& sq) {
+  const Hp& h = v.h;
+  const int W = v.W;
+  const bool vec_ok = T->vec_ok != 0;
+  switch (v.kind) {
+    case 0: run_chunk<0, false, NT>(tid, h, shards, W, T->p, T->s0, T->s1, begin, count, vec_ok, sq); break;
+    case 1: run_chunk<0, true, NT>(tid, h, shards, W, T->p, T->s0, T->s1, begin, count, vec_ok, sq); break;
+    case 2: run_chunk<1, false, NT>(tid, h, shards, W, T->p, T->s0, T->s1, begin, count, vec_ok, sq); break;
+    default: run_chunk<1, true, NT>(tid, h, shards, W, T->p, T->s0, T->s1, begin, count, vec_ok, sq); break;
+  }
+}
+
 template <int NT>
 __device__ __forceinline__ void run_chunk_any(unsigned int tid, const PsJobDev* J, const PsTaskDev* T,
                                               const void* const* shards, size_t begin, unsigned int count,
@@ -289,21 +317,39 @@ __device__ __forceinline__ void run_chunk_any(unsigned int tid, const PsJobDev* 
   }
 }
 
+// Sum of n partial sums of squares in a FIXED order, by one warp: lane l adds
+// the partials l, l+32, l+64, ... in increasing order, then the lanes are
+// combined by a shuffle tree.  The result does not depend on which CTA produced
+// which partial nor on arrival order.  (A single thread walking the list costs
+// one L2 round trip per few partials: about 10 us for the 576 chunks of a
+// 590 K-element tensor, which was most of such a launch's duration.)
+__device__ __forceinline__ double sum_partials_warp(const double* partials, unsigned int n, unsigned int lane) {
+  double tot = 0.0;
+  for (unsigned int k = lane; k < n; k += 32) tot += __ldcg(partials + k);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) tot += __shfl_down_sync(0xffffffffu, tot, o);
+  return tot;     // complete in lane 0
+}
+
 // Publishes one partial sum of squares of a chunk (slot = chunk * parts + part)
-// and, for the caller that delivers the task's last partial, adds all of the
-// task's partials in slot order: the per-block norm does not depend on which
-// CTA ran which chunk nor on arrival order.  One thread per partial calls this.
+// and, in the warp that delivers the task's last partial, adds all of the
+// task's partials in the fixed order above.  Called by all 32 lanes of one warp
+// per partial; `s` is taken from lane 0.
 __device__ __forceinline__ void publish_part(PsTaskDev* tasks, unsigned int t, unsigned int slot, unsigned int parts,
-                                             double s, PsStat* stats, double* partials) {
+                                             double s, PsStat* stats, double* partials, unsigned int lane) {
   const PsTaskDev* T = tasks + t;
   const unsigned int first = T->first_chunk * parts, n = T->nchunks * parts;
-  __stcg(partials + slot, s);
-  __threadfence();
-  const unsigned int done = atomicAdd(&tasks[t].ticket, 1u);
-  if (done == n - 1) {
+  unsigned int done = 0;
+  if (lane == 0) {
+    __stcg(partials + slot, s);
     __threadfence();
-    double tot = 0.0;
-    for (unsigned int k = 0; k < n; ++k) tot += __ldcg(partials + first + k);
+    done = atomicAdd(&tasks[t].ticket, 1u);
+    __threadfence();
+  }
+  done = __shfl_sync(0xffffffffu, done, 0);
+  if (done != n - 1) return;
+  const double tot = sum_partials_warp(partials + first, n, lane);
+  if (lane == 0) {
     PsStat st;
     st.sqnorm = tot;
     st.step = T->step;
@@ -329,6 +375,38 @@ __device__ __forceinline__ void profile_chunk(PsTaskDev* T, unsigned long long t
   atomicMin(&T->t_first, t0);
   atomicMax(&T->t_last, t1);
 }
+
+// Completion signal of a launch.  Every thread of a CTA calls this when the CTA
+// has no more work.  The CTA that leaves last (counted in *exited, which it
+// clears for the next launch that uses the same counter) stores `seq` to
+// *done_word — a word in page-locked host memory that the host polls instead of
+// recording and querying an event per launch.
+// Ordering: the barrier puts the CTA's stores before thread 0's fence, which is
+// cumulative, so they are visible device-wide before the CTA is counted; the
+// last CTA's own fence does the same for the counts it has seen before it
+// issues the store.  Whoever acts on the word is a later launch on this device
+// (or a copy engine reading device memory), for which device-wide visibility is
+// what counts; a system-wide fence here cost 1.4 us of every small launch
+// (measured) and bought nothing for such readers.
+// done_word == nullptr: the launch does not signal.
+__device__ __forceinline__ void signal_exit(unsigned int* exited, unsigned long long* done_word,
+                                            unsigned long long seq) {
+  if (!done_word) return;
+  __syncthreads();
+  if (threadIdx.x != 0) return;
+  __threadfence();
+  if (atomicAdd(exited, 1u) != gridDim.x - 1) return;
+  *exited = 0;
+  __threadfence();
+  *reinterpret_cast<volatile unsigned long long*>(done_word) = seq;
+}
+
+// Programmatic dependent launch: lets the next launch of the stream start its
+// prologue while this one runs (a no-op for launches without the attribute) ...
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+// ... and waits until the launches this one depends on have completed and their
+// stores are visible (returns at once when there is no such dependency).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // Advances `cursor` (uniform in the calling warp) to the task that owns chunk
 // idx: starts[] is increasing and starts[cursor] <= idx on entry.

@@ -27,9 +27,9 @@
 namespace psb {
 
 constexpr uint32_t kMagic = 0x50534232u;   // "PSB2"
-constexpr int kSlots = 8;                  // task tables in flight
+constexpr int kSlots = 16;                 // task tables in flight
 constexpr int kInlineGridFactor = 4;         // an inline launch has at most this many CTAs per resident slot
-constexpr int kWorkStreams = 4;             // overlap mode: launches rotate over this many streams
+constexpr int kWorkStreams = 8;             // overlap mode: launches rotate over this many streams
 constexpr unsigned int kMaxChunk = 1u << 20;
 
 struct Job {
@@ -91,11 +91,16 @@ struct Slot {
   double* partials = nullptr;
   size_t partial_cap = 0;
   PsTaskMut* mut = nullptr;                // per-task state of launches whose table travels as a kernel parameter
-  cudaEvent_t done = nullptr;
+  cudaEvent_t done = nullptr;              // marks a point of `stream` at or after the slot's launch
+  bool done_recorded = false;              // ... once it has been recorded (lazily for launches that signal)
   cudaEvent_t copied = nullptr;            // table upload finished (recorded on the copy stream)
   cudaEvent_t input = nullptr;             // overlap mode: the caller's stream at the time of the call
   bool inflight = false;
   unsigned long long gen = 0;
+  unsigned long long seq = 0;              // number of the slot's launch (what its kernel stores when it has finished)
+  bool signals = false;                    // the kernel stores seq to the slot's completion word
+  cudaStream_t stream = nullptr;           // the stream the launch went to
+  int work_stream = -1;                    // its index among the service's streams, -1 = a caller's stream
 };
 
 struct Plan {                              // one built task table (host copy)
@@ -103,7 +108,10 @@ struct Plan {                              // one built task table (host copy)
   std::vector<int> order;                  // block indices in table order
   unsigned int total_chunks = 0, chunk_elems = 0;
   bool has_sparse = false;                 // some task carries row-sparse shards (direct-load kernel only)
+  unsigned long long algo_bytes = 0;       // algorithmic bytes of the launch (dense semantics)
 };
+
+enum { kVarLdg = 0, kVarInline = 1, kVarBulk = 2, kVariants = 3 };
 
 }  // namespace psb
 
@@ -132,11 +140,24 @@ struct ps_service {
   cudaStream_t copy_stream = nullptr;      // table uploads run here, beside the previous launch
   cudaStream_t work_streams[kWorkStreams] = {};   // overlap mode: launches rotate over these
   int next_work = 0;
-  unsigned int unjoined = 0;               // overlap mode: slots whose launch no caller stream has joined yet
+  // overlap mode: per service stream, the slot of its latest launch and that launch's number,
+  // and the number of the latest launch a caller's stream has joined (ps_join)
+  int ws_last_slot[kWorkStreams] = {};
+  unsigned long long ws_last_seq[kWorkStreams] = {}, ws_joined_seq[kWorkStreams] = {};
   long long opt_overlap = 0;
   long long opt_inline = 1;               // small launches carry their table as a kernel parameter
+  long long opt_pdl = 1;                  // small launches are launched with programmatic stream serialization
   int occ_ctas = 0;
   unsigned long long launches = 0;
+  unsigned long long var_launches[kVariants] = {}, var_bytes[kVariants] = {};
+  // completion words, one per slot, in page-locked host memory: the kernel of a slot's launch
+  // stores the launch number there when its last CTA leaves
+  volatile unsigned long long* done_host = nullptr;
+  unsigned long long* done_dev = nullptr;  // the same words as the device addresses them
+  unsigned int* exit_ctrs = nullptr;       // device, one CTA counter per slot (inline launches), all-zero between launches
+  Plan plan;                               // scratch reused by every ps_aggregate
+  std::vector<int> idx;                    // the same for the validated ready list
+  std::vector<int> free_blocks;            // entries of `blocks` released by ps_unregister_block
   int last_grid = 0, last_block = 0;
   const char* last_kernel = "none";
   std::string cuda_err;
@@ -288,14 +309,17 @@ constexpr unsigned int kChunkAuto = 8192, kChunkFloor = 1024;
 
 // A launch with fewer chunks than resident CTAs leaves SMs idle while each busy
 // CTA streams a whole chunk at single-CTA bandwidth (about 19 us for 8192
-// elements, measured): such small launches get smaller chunks, halving until
-// every resident CTA has one or the floor is reached.
+// elements, measured): such small launches get smaller chunks, halving as long
+// as the chunks still fit ONE wave of resident CTAs or until the floor is
+// reached.  One wave of CTAs with two or four vectors per thread beats two or
+// four waves of CTAs with one: every CTA pays its fixed cost (start, task lookup,
+// the latency of its first loads, the reduction of the norm, the ticket) once.
 unsigned int auto_chunk(ps_service* s, const std::vector<int>& idx, int grid) {
   unsigned int ce = kChunkAuto;
   while (ce > kChunkFloor) {
     unsigned long long chunks = 0;
-    for (int bi : idx) chunks += (s->blocks[bi].nelem + ce - 1) / ce;
-    if (chunks >= (unsigned long long)grid) break;
+    for (int bi : idx) chunks += (s->blocks[bi].nelem + ce / 2 - 1) / (ce / 2);
+    if (chunks > (unsigned long long)grid) break;
     ce >>= 1;
   }
   return ce;
@@ -406,6 +430,8 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
     if (chunk > 0xfffffff0ull) return PS_ERR_BAD_ARG;
   }
   plan->total_chunks = (unsigned int)chunk;
+  plan->algo_bytes = 0;
+  for (int bi : plan->order) plan->algo_bytes += s->blocks[bi].nelem * bytes_per_elem(s->jobs[s->blocks[bi].job]);
   PsTableHdr* h = reinterpret_cast<PsTableHdr*>(base);
   h->counter = 0;
   h->n_tasks = (unsigned int)n;
@@ -417,19 +443,45 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
   h->parts_per_chunk = (use_bulk(s) && !plan->has_sparse) ? kBulkConsumerWarps : 1;
   h->profile = s->opt_profile ? 1u : 0u;
   h->sparse_off = (unsigned int)sparse_off;
+  h->exited = 0;
+  return PS_OK;
+}
+
+// Has the slot's launch finished?  Launches that signal are checked by reading
+// their completion word (no driver call); the others by querying their event.
+bool slot_finished(ps_service* s, Slot& sl) {
+  if (!sl.inflight) return true;
+  const int i = (int)(&sl - s->slots);
+  if (sl.signals && s->done_host[i] == sl.seq) { sl.inflight = false; return true; }
+  if (sl.done_recorded && cudaEventQuery(sl.done) == cudaSuccess) { sl.inflight = false; return true; }
+  return false;
+}
+
+// An event at or after the slot's launch exists on its stream after this call.
+int ensure_done_event(ps_service* s, Slot& sl) {
+  if (sl.done_recorded) return PS_OK;
+  PS_CUDA(s, cudaEventRecord(sl.done, sl.stream));
+  sl.done_recorded = true;
+  return PS_OK;
+}
+
+// Blocks the host until the slot's launch has finished.
+int wait_slot(ps_service* s, Slot& sl) {
+  if (slot_finished(s, sl)) return PS_OK;
+  int rc = ensure_done_event(s, sl);
+  if (rc) return rc;
+  PS_CUDA(s, cudaEventSynchronize(sl.done));
+  sl.inflight = false;
   return PS_OK;
 }
 
 int acquire_slot(ps_service* s, size_t table_bytes, size_t nchunks, Slot** out) {
   Slot& sl = s->slots[s->next_slot];
-  if (sl.inflight) {
-    PS_CUDA(s, cudaEventSynchronize(sl.done));
-    sl.inflight = false;
-  }
+  int rc = wait_slot(s, sl);
+  if (rc) return rc;
   if (!sl.done) PS_CUDA(s, cudaEventCreateWithFlags(&sl.done, cudaEventDisableTiming));
   if (!sl.copied) PS_CUDA(s, cudaEventCreateWithFlags(&sl.copied, cudaEventDisableTiming));
   if (!sl.input) PS_CUDA(s, cudaEventCreateWithFlags(&sl.input, cudaEventDisableTiming));
-  s->unjoined &= ~(1u << (unsigned)(&sl - s->slots));   // its previous launch has completed (host waited)
   if (table_bytes > sl.cap) {
     size_t ncap = std::max<size_t>(table_bytes * 2, 1 << 16);
     if (sl.host) PS_CUDA(s, cudaFreeHost(sl.host));
@@ -456,17 +508,30 @@ int acquire_slot(ps_service* s, size_t table_bytes, size_t nchunks, Slot** out) 
   return PS_OK;
 }
 
+// The slot of the block's last launch if that launch may still be running, else nullptr.
+Slot* pending_slot(ps_service* s, Block& b) {
+  if (b.last_slot < 0) return nullptr;
+  Slot& sl = s->slots[b.last_slot];
+  if (sl.gen != b.last_slot_gen || slot_finished(s, sl)) return nullptr;
+  return &sl;
+}
+
 // Makes `stream` wait for everything enqueued so far that touches block b.
 // `waited` (optional) collects the slots this call has already made `stream`
 // wait for, so that a list of many blocks from one earlier launch costs one wait.
+// A launch that went to `stream` itself needs no wait: stream order covers it.
 int order_after_block(ps_service* s, Block& b, cudaStream_t stream, unsigned int* waited = nullptr) {
-  if (b.last_slot >= 0) {
-    Slot& sl = s->slots[b.last_slot];
+  if (Slot* sl = pending_slot(s, b)) {
     const unsigned int bit = 1u << (unsigned)b.last_slot;
-    if (sl.inflight && sl.gen == b.last_slot_gen && !(waited && (*waited & bit))) {
-      PS_CUDA(s, cudaStreamWaitEvent(stream, sl.done, 0));
-      if (waited) *waited |= bit;
+    // (a caller's stream handle may have been destroyed and handed out again, so only
+    // the service's own streams are trusted to be the same stream when the handles match)
+    const bool same = sl->work_stream >= 0 && sl->stream == stream;
+    if (!same && !(waited && (*waited & bit))) {
+      int rc = ensure_done_event(s, *sl);
+      if (rc) return rc;
+      PS_CUDA(s, cudaStreamWaitEvent(stream, sl->done, 0));
     }
+    if (waited) *waited |= bit;
   }
   if (b.mig_batch >= 0) {
     bool ready = false;
@@ -486,16 +551,37 @@ int order_after_block(ps_service* s, Block& b, cudaStream_t stream, unsigned int
   return PS_OK;
 }
 
-int push_checked(ps_service* s, int job, int block, int worker, const void* ptr, Block** out) {
+// in_place: the kernel will read `ptr` itself (false: ps_push_host copies it to aligned staging first)
+int push_checked(ps_service* s, int job, int block, int worker, const void* ptr, Block** out, bool in_place = true) {
   const int bi = find_block(s, job, block);
   if (bi < 0 || !ptr) return PS_ERR_BAD_ARG;
   Block& b = s->blocks[bi];
   const Job& j = s->jobs[b.job];
   if (worker < 0 || worker >= j.d.num_workers) return PS_ERR_BAD_ARG;
   if (reinterpret_cast<uintptr_t>(ptr) & (j.grad_esize() - 1)) return PS_ERR_ALIGN;
+  // a block with row-sparse pushes is streamed row by row with 128-bit loads from
+  // every shard, the dense ones included: those need 16-byte aligned starts
+  if (in_place && b.nsparse > 0 && (reinterpret_cast<uintptr_t>(ptr) & 15u)) return PS_ERR_ALIGN;
   if (b.pushed[worker]) return PS_ERR_DUPLICATE;
   *out = &b;
   return PS_OK;
+}
+
+// Launches one aggregation kernel with an optional programmatic-serialization attribute.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t stream,
+                                 bool pdl, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 }  // namespace
@@ -522,6 +608,19 @@ int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes
       e = cudaStreamCreateWithFlags(&s->work_streams[i], cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaMalloc(&s->status_dev, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(s->status_dev, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc(&s->exit_ctrs, kSlots * sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(s->exit_ctrs, 0, kSlots * sizeof(unsigned int));
+    if (e == cudaSuccess) {
+      void* h = nullptr;
+      e = cudaHostAlloc(&h, kSlots * sizeof(unsigned long long), cudaHostAllocMapped);
+      if (e == cudaSuccess) {
+        std::memset(h, 0, kSlots * sizeof(unsigned long long));
+        s->done_host = static_cast<volatile unsigned long long*>(h);
+        void* d = nullptr;
+        e = cudaHostGetDevicePointer(&d, h, 0);
+        s->done_dev = static_cast<unsigned long long*>(d);
+      }
+    }
     if (e == cudaSuccess) e = cudaStreamSynchronize(cudaStreamLegacy);
     for (int c = 0; e == cudaSuccess && c < num_contexts; ++c) {
       void* base = nullptr;
@@ -532,6 +631,8 @@ int ps_create(ps_service** out, int device, int num_contexts, size_t arena_bytes
       const bool oom = (e == cudaErrorMemoryAllocation);
       for (auto& c : s->ctxs) if (c.base) cudaFree(c.base);
       if (s->status_dev) cudaFree(s->status_dev);
+      if (s->exit_ctrs) cudaFree(s->exit_ctrs);
+      if (s->done_host) cudaFreeHost(const_cast<unsigned long long*>(s->done_host));
       if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
       for (auto ws : s->work_streams) if (ws) cudaStreamDestroy(ws);
       cudaGetLastError();
@@ -565,6 +666,8 @@ int ps_destroy(ps_service* s) {
     if (s->jobs_dev) cudaFree(s->jobs_dev);
     if (s->stats_dev) cudaFree(s->stats_dev);
     if (s->status_dev) cudaFree(s->status_dev);
+    if (s->exit_ctrs) cudaFree(s->exit_ctrs);
+    if (s->done_host) cudaFreeHost(const_cast<unsigned long long*>(s->done_host));
     if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
     for (auto ws : s->work_streams) if (ws) cudaStreamDestroy(ws);
   }
@@ -617,16 +720,21 @@ int ps_register_block(ps_service* s, int job, int block, size_t nelem, int ctx, 
   b.pushed.assign(j.d.num_workers, nullptr);
   b.row_ids.assign(j.d.num_workers, nullptr);
   b.row_cnt.assign(j.d.num_workers, 0);
-  b.stat_idx = (unsigned int)s->blocks.size();
+  // an entry released by ps_unregister_block is used again (with its statistics record), so
+  // blocks that come and go, e.g. by migration between services, do not grow the tables
+  const bool reuse = !s->free_blocks.empty();
+  const size_t bi_new = reuse ? (size_t)s->free_blocks.back() : s->blocks.size();
+  b.stat_idx = (unsigned int)bi_new;
   if (has_device(s)) PS_CUDA(s, cudaSetDevice(s->device));
   int rc = arena_alloc(s, ctx, b.bytes, &b.off);
   if (rc) return rc;
   if (has_device(s)) {
-    rc = grow_dev(s, &s->stats_dev, &s->stats_dev_cap, s->blocks.size() + 1, true);
+    rc = grow_dev(s, &s->stats_dev, &s->stats_dev_cap, bi_new + 1, true);
     cudaError_t e = cudaSuccess;
     if (!rc) {
       char* base = s->ctxs[ctx].base + b.off;
       e = cudaMemset(base, 0, b.bytes);
+      if (e == cudaSuccess && reuse) e = cudaMemset(s->stats_dev + bi_new, 0, sizeof(PsStat));
       if (e == cudaSuccess && init) e = cudaMemcpy(base, init, nelem * sizeof(float), cudaMemcpyDefault);
       // a device memset may return before it has run, and the service's streams do not
       // synchronize with the default stream: wait here, once per registration
@@ -636,8 +744,13 @@ int ps_register_block(ps_service* s, int job, int block, size_t nelem, int ctx, 
     if (rc) { s->ctxs[ctx].arena.release(b.off, b.bytes); return rc; }
   }
   if (block >= (int)j.block_of_id.size()) j.block_of_id.resize(block + 1, -1);
-  j.block_of_id[block] = (int)s->blocks.size();
-  s->blocks.push_back(std::move(b));
+  j.block_of_id[block] = (int)bi_new;
+  if (reuse) {
+    s->free_blocks.pop_back();
+    s->blocks[bi_new] = std::move(b);
+  } else {
+    s->blocks.push_back(std::move(b));
+  }
   return PS_OK;
 }
 
@@ -702,6 +815,9 @@ static int push_rows_locked(ps_service* s, int job, int block, int worker, const
       (reinterpret_cast<uintptr_t>(row_ids) & 3u))
     return PS_ERR_ALIGN;
   if (b.pushed[worker]) return PS_ERR_DUPLICATE;
+  // the dense shards this block already holds will be read with 128-bit loads too
+  for (int w = 0; w < j.d.num_workers; ++w)
+    if (b.pushed[w] && !b.row_ids[w] && (reinterpret_cast<uintptr_t>(b.pushed[w]) & 15u)) return PS_ERR_ALIGN;
   b.pushed[worker] = values;
   b.row_ids[worker] = row_ids;
   b.row_cnt[worker] = (unsigned int)n_rows;
@@ -711,10 +827,16 @@ static int push_rows_locked(ps_service* s, int job, int block, int worker, const
   return PS_OK;
 }
 
-int ps_push_batch(ps_service* s, int n, const int* jobs, const int* blocks, const int* workers,
-                  const void* const* ptrs) {
-  if (!alive(s)) return PS_ERR_BAD_HANDLE;
-  std::lock_guard<std::mutex> lk(s->mu);
+static void unpush_locked(ps_service* s, int n, const int* jobs, const int* blocks, const int* workers) {
+  for (int i = 0; i < n; ++i) {
+    Block& b = s->blocks[find_block(s, jobs[i], blocks[i])];
+    b.pushed[workers[i]] = nullptr;
+    b.npushed--;
+  }
+}
+
+static int push_batch_locked(ps_service* s, int n, const int* jobs, const int* blocks, const int* workers,
+                             const void* const* ptrs) {
   if (n < 0 || (n > 0 && (!jobs || !blocks || !workers || !ptrs))) return PS_ERR_BAD_ARG;
   int rc = PS_OK, done = 0;
   for (; done < n; ++done) {
@@ -724,21 +846,22 @@ int ps_push_batch(ps_service* s, int n, const int* jobs, const int* blocks, cons
     b->pushed[workers[done]] = ptrs[done];
     b->npushed++;
   }
-  if (rc) {   // roll back: all-or-nothing
-    for (int i = 0; i < done; ++i) {
-      Block& b = s->blocks[find_block(s, jobs[i], blocks[i])];
-      b.pushed[workers[i]] = nullptr;
-      b.npushed--;
-    }
-  }
+  if (rc) unpush_locked(s, done, jobs, blocks, workers);   // all-or-nothing
   return rc;
+}
+
+int ps_push_batch(ps_service* s, int n, const int* jobs, const int* blocks, const int* workers,
+                  const void* const* ptrs) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  return push_batch_locked(s, n, jobs, blocks, workers, ptrs);
 }
 
 int ps_push_host(ps_service* s, int job, int block, int worker, const void* host_ptr, void* stream) {
   if (!alive(s)) return PS_ERR_BAD_HANDLE;
   std::lock_guard<std::mutex> lk(s->mu);
   Block* b = nullptr;
-  int rc = push_checked(s, job, block, worker, host_ptr, &b);
+  int rc = push_checked(s, job, block, worker, host_ptr, &b, false);
   if (rc) return rc;
   if (!has_device(s)) return PS_ERR_NO_DEVICE;
   PS_CUDA(s, cudaSetDevice(s->device));
@@ -766,19 +889,13 @@ int ps_push_host(ps_service* s, int job, int block, int worker, const void* host
   return PS_OK;
 }
 
-int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_) {
-  if (!alive(s)) return PS_ERR_BAD_HANDLE;
-  std::lock_guard<std::mutex> lk(s->mu);
-  std::vector<int> idx;
-  int rc = validate_ready(s, ready, n_ready, &idx);
-  if (rc) return rc;
-  if (!has_device(s)) return PS_ERR_NO_DEVICE;
-  if (idx.empty()) return PS_OK;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+// Aggregates the validated blocks s->idx in one launch.  The service lock is held.
+static int aggregate_locked(ps_service* s, cudaStream_t stream, unsigned int flags) {
+  const std::vector<int>& idx = s->idx;
   PS_CUDA(s, cudaSetDevice(s->device));
   ++s->call_id;
-  Plan plan;
-  rc = build_plan(s, idx, &plan);
+  Plan& plan = s->plan;
+  int rc = build_plan(s, idx, &plan);
   if (rc) return rc;
   Slot* sl = nullptr;
   const bool bulk = use_bulk(s) && !plan.has_sparse;
@@ -793,24 +910,41 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
   // Overlap mode: the launch goes to one of the service-owned streams, after the
   // work the caller has enqueued on `stream` so far; consecutive launches then
   // overlap (the next one's CTAs fill the SMs the previous one's tail leaves idle).
+  // A launch that has to follow an unfinished one (a block aggregated again) goes to
+  // that launch's stream, where stream order is the dependency: no event.
   cudaStream_t run = stream;
+  int ws = -1;
   if (s->opt_overlap) {
-    run = s->work_streams[s->next_work];
-    s->next_work = (s->next_work + 1) % kWorkStreams;
-    PS_CUDA(s, cudaEventRecord(sl->input, stream));
-    PS_CUDA(s, cudaStreamWaitEvent(run, sl->input, 0));
+    for (int bi : idx) {
+      Slot* dep = pending_slot(s, s->blocks[bi]);
+      if (dep && dep->work_stream >= 0) { ws = dep->work_stream; break; }
+    }
+    if (ws < 0) {
+      ws = s->next_work;
+      s->next_work = (s->next_work + 1) % kWorkStreams;
+    }
+    run = s->work_streams[ws];
+    if (!(flags & PS_ROUND_INPUTS_COMPLETE)) {
+      PS_CUDA(s, cudaEventRecord(sl->input, stream));
+      PS_CUDA(s, cudaStreamWaitEvent(run, sl->input, 0));
+    }
   }
   unsigned int waited = 0;
   for (int bi : idx) {
     rc = order_after_block(s, s->blocks[bi], run, &waited);
     if (rc) return rc;
   }
+  const unsigned long long seq = s->launches + 1;
+  unsigned long long* done_word = s->done_dev + slot_index;
   int grid = (int)std::min<unsigned long long>(plan.total_chunks, (unsigned long long)grid_cap(s));
+  cudaError_t le;
   if (inl) {
     PsInlineTable tbl;
     std::memcpy(tbl.bytes, plan.bytes.data(), plan.bytes.size());
     grid = (int)plan.total_chunks;
-    ps_aggregate_inline_kernel<<<grid, kThreads, 0, run>>>(tbl, s->jobs_dev, s->stats_dev, sl->partials, sl->mut);
+    le = launch_kernel(ps_aggregate_inline_kernel, grid, kThreads, 0, run, s->opt_pdl != 0, tbl,
+                       (const PsJobDev*)s->jobs_dev, s->stats_dev, sl->partials, sl->mut, s->exit_ctrs + slot_index,
+                       done_word, seq);
   } else {
     std::memcpy(sl->host, plan.bytes.data(), plan.bytes.size());
     // The table depends on nothing the caller enqueued, so its upload goes to the
@@ -819,17 +953,39 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
     PS_CUDA(s, cudaEventRecord(sl->copied, s->copy_stream));
     PS_CUDA(s, cudaStreamWaitEvent(run, sl->copied, 0));
     if (bulk)
-      ps_aggregate_bulk_kernel<<<grid, kBulkThreads, kBulkSmemBytes, run>>>(sl->dev, s->jobs_dev, s->stats_dev,
-                                                                            sl->partials, s->status_dev);
+      le = launch_kernel(ps_aggregate_bulk_kernel, grid, kBulkThreads, kBulkSmemBytes, run, false, sl->dev,
+                         (const PsJobDev*)s->jobs_dev, s->stats_dev, sl->partials, s->status_dev);
     else
-      ps_aggregate_ldg_kernel<<<grid, kThreads, 0, run>>>(sl->dev, s->jobs_dev, s->stats_dev, sl->partials);
+      le = launch_kernel(ps_aggregate_ldg_kernel, grid, kThreads, 0, run, false, sl->dev,
+                         (const PsJobDev*)s->jobs_dev, s->stats_dev, sl->partials, done_word, seq);
   }
-  PS_CUDA(s, cudaGetLastError());
-  PS_CUDA(s, cudaEventRecord(sl->done, run));
+  if (le != cudaSuccess) {
+    s->cuda_err = std::string("kernel launch: ") + cudaGetErrorString(le);
+    cudaGetLastError();
+    return PS_ERR_CUDA;
+  }
+  sl->seq = seq;
+  sl->signals = !bulk;
+  sl->stream = run;
+  sl->work_stream = ws;
+  sl->done_recorded = false;
   sl->inflight = true;
-  if (s->opt_overlap) s->unjoined |= 1u << (unsigned)slot_index;
+  // A launch on a caller's stream is marked at once (the handle may not outlive the
+  // call); so is one whose kernel does not signal.  The others get their event only
+  // if some other stream ever has to wait for them.
+  if (ws < 0 || !sl->signals) {
+    PS_CUDA(s, cudaEventRecord(sl->done, run));
+    sl->done_recorded = true;
+  }
+  if (ws >= 0) {
+    s->ws_last_slot[ws] = slot_index;
+    s->ws_last_seq[ws] = seq;
+  }
   s->next_slot = (s->next_slot + 1) % kSlots;
-  s->launches++;
+  s->launches = seq;
+  const int var = inl ? kVarInline : bulk ? kVarBulk : kVarLdg;
+  s->var_launches[var]++;
+  s->var_bytes[var] += plan.algo_bytes;
   s->last_grid = grid;
   s->last_block = bulk ? kBulkThreads : kThreads;
   s->last_kernel = inl ? "inline" : bulk ? "bulk" : "ldg";
@@ -848,27 +1004,67 @@ int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_
   return PS_OK;
 }
 
+int ps_aggregate(ps_service* s, const ps_task* ready, int n_ready, void* stream_) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  int rc = validate_ready(s, ready, n_ready, &s->idx);
+  if (rc) return rc;
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  if (s->idx.empty()) return PS_OK;
+  return aggregate_locked(s, static_cast<cudaStream_t>(stream_), 0u);
+}
+
+static int push_batch_locked(ps_service* s, int n, const int* jobs, const int* blocks, const int* workers,
+                             const void* const* ptrs);
+static void unpush_locked(ps_service* s, int n, const int* jobs, const int* blocks, const int* workers);
+
+int ps_round(ps_service* s, int n_push, const int* jobs, const int* blocks, const int* workers,
+             const void* const* grad_dev_ptrs, const ps_task* ready, int n_ready, unsigned int flags, void* stream_,
+             const float** params_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (flags & ~(unsigned int)PS_ROUND_INPUTS_COMPLETE) return PS_ERR_BAD_ARG;
+  int rc = push_batch_locked(s, n_push, jobs, blocks, workers, grad_dev_ptrs);
+  if (rc) return rc;
+  rc = validate_ready(s, ready, n_ready, &s->idx);
+  if (!rc && !has_device(s)) rc = PS_ERR_NO_DEVICE;
+  if (!rc && !s->idx.empty()) rc = aggregate_locked(s, static_cast<cudaStream_t>(stream_), flags);
+  if (rc) {
+    unpush_locked(s, n_push, jobs, blocks, workers);
+    return rc;
+  }
+  if (params_out)
+    for (size_t i = 0; i < s->idx.size(); ++i) params_out[i] = blk_p(s, s->blocks[s->idx[i]]);
+  return PS_OK;
+}
+
 int ps_join(ps_service* s, void* stream_) {
   if (!alive(s)) return PS_ERR_BAD_HANDLE;
   std::lock_guard<std::mutex> lk(s->mu);
   if (!has_device(s)) return PS_OK;
   PS_CUDA(s, cudaSetDevice(s->device));
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  for (int i = 0; i < kSlots; ++i) {
-    if (!(s->unjoined & (1u << i))) continue;
-    if (s->slots[i].inflight) PS_CUDA(s, cudaStreamWaitEvent(stream, s->slots[i].done, 0));
+  // per service stream: its launches finish in order, so the latest one stands for all
+  for (int w = 0; w < kWorkStreams; ++w) {
+    if (s->ws_last_seq[w] == s->ws_joined_seq[w]) continue;
+    s->ws_joined_seq[w] = s->ws_last_seq[w];
+    Slot& sl = s->slots[s->ws_last_slot[w]];
+    if (sl.seq != s->ws_last_seq[w] || slot_finished(s, sl)) continue;   // recycled (so finished) or finished
+    int rc = ensure_done_event(s, sl);
+    if (rc) return rc;
+    PS_CUDA(s, cudaStreamWaitEvent(stream, sl.done, 0));
   }
-  s->unjoined = 0;
   return PS_OK;
 }
 
 int ps_plan(ps_service* s, const ps_task* ready, int n_ready, ps_chunk_info* out, size_t cap, size_t* n_out) {
   if (!alive(s)) return PS_ERR_BAD_HANDLE;
   std::lock_guard<std::mutex> lk(s->mu);
-  std::vector<int> idx;
+  std::vector<int>& idx = s->idx;
   int rc = validate_ready(s, ready, n_ready, &idx);
   if (rc) return rc;
-  Plan plan;
+  Plan& plan = s->plan;
+  plan.total_chunks = 0;
   if (!idx.empty()) {
     rc = build_plan(s, idx, &plan);
     if (rc) return rc;
@@ -1116,9 +1312,9 @@ int ps_unregister_block(ps_service* s, int job, int block) {
     PS_CUDA(s, cudaSetDevice(s->device));
     ++s->call_id;
     // everything this service enqueued for the block: its last launch, its last copy
-    if (b.last_slot >= 0) {
-      Slot& sl = s->slots[b.last_slot];
-      if (sl.inflight && sl.gen == b.last_slot_gen) PS_CUDA(s, cudaEventSynchronize(sl.done));
+    if (Slot* sl = pending_slot(s, b)) {
+      int rc = wait_slot(s, *sl);
+      if (rc) return rc;
     }
     if (b.mig_batch >= 0) {
       bool ready = false;
@@ -1136,6 +1332,7 @@ int ps_unregister_block(ps_service* s, int job, int block) {
   b.nelem = 0;
   b.bytes = 0;
   b.npushed = 0;
+  s->free_blocks.push_back(bi);
   return PS_OK;
 }
 
@@ -1150,8 +1347,10 @@ int ps_block_stats(ps_service* s, int job, int block, double* sq_out, unsigned l
   *sq_out = 0.0;
   if (!has_device(s) || b.last_slot < 0) return PS_OK;
   PS_CUDA(s, cudaSetDevice(s->device));
-  Slot& sl = s->slots[b.last_slot];
-  if (sl.inflight && sl.gen == b.last_slot_gen) PS_CUDA(s, cudaEventSynchronize(sl.done));
+  if (Slot* sl = pending_slot(s, b)) {
+    int rc = wait_slot(s, *sl);
+    if (rc) return rc;
+  }
   PsStat st;
   PS_CUDA(s, cudaMemcpy(&st, s->stats_dev + b.stat_idx, sizeof st, cudaMemcpyDeviceToHost));
   *sq_out = st.sqnorm;
@@ -1163,8 +1362,10 @@ static int read_stat(ps_service* s, Block& b, PsStat* st) {
   std::memset(st, 0, sizeof *st);
   if (!has_device(s) || b.last_slot < 0) return PS_OK;
   PS_CUDA(s, cudaSetDevice(s->device));
-  Slot& sl = s->slots[b.last_slot];
-  if (sl.inflight && sl.gen == b.last_slot_gen) PS_CUDA(s, cudaEventSynchronize(sl.done));
+  if (Slot* sl = pending_slot(s, b)) {
+    int rc = wait_slot(s, *sl);
+    if (rc) return rc;
+  }
   PS_CUDA(s, cudaMemcpy(st, s->stats_dev + b.stat_idx, sizeof *st, cudaMemcpyDeviceToHost));
   return PS_OK;
 }
@@ -1246,6 +1447,9 @@ int ps_set_option(ps_service* s, int option, long long value) {
     case PS_OPT_INLINE_TABLE:
       s->opt_inline = value ? 1 : 0;
       return PS_OK;
+    case PS_OPT_PDL:
+      s->opt_pdl = value ? 1 : 0;
+      return PS_OK;
     default:
       return PS_ERR_BAD_ARG;
   }
@@ -1263,6 +1467,7 @@ int ps_get_option(ps_service* s, int option, long long* out) {
     case PS_OPT_PROFILE: *out = s->opt_profile; return PS_OK;
     case PS_OPT_OVERLAP: *out = s->opt_overlap; return PS_OK;
     case PS_OPT_INLINE_TABLE: *out = s->opt_inline; return PS_OK;
+    case PS_OPT_PDL: *out = s->opt_pdl; return PS_OK;
     default: return PS_ERR_BAD_ARG;
   }
 }
@@ -1277,6 +1482,15 @@ int ps_arena_info(ps_service* s, int ctx, size_t* used_out, size_t* largest_free
   }
   if (used_out) *used_out = s->ctxs[ctx].arena.used();
   if (largest_free_out) *largest_free_out = s->ctxs[ctx].arena.largest_free();
+  return PS_OK;
+}
+
+int ps_registry_info(ps_service* s, size_t* jobs_out, size_t* blocks_out, size_t* block_entries_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (jobs_out) *jobs_out = s->jobs.size();
+  if (blocks_out) *blocks_out = s->blocks.size() - s->free_blocks.size();
+  if (block_entries_out) *block_entries_out = s->blocks.size();
   return PS_OK;
 }
 
@@ -1313,6 +1527,19 @@ int ps_launch_info(ps_service* s, unsigned long long* launches, int* grid, int* 
   if (grid) *grid = s->last_grid;
   if (block) *block = s->last_block;
   if (name) *name = s->last_kernel;
+  return PS_OK;
+}
+
+int ps_launch_stats(ps_service* s, int variant, unsigned long long* launches_out, unsigned long long* bytes_out,
+                    const char** name_out) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (variant < 0 || variant >= kVariants) return PS_ERR_BAD_ARG;
+  static const char* const names[kVariants] = {"ps_aggregate_ldg_kernel", "ps_aggregate_inline_kernel",
+                                               "ps_aggregate_bulk_kernel"};
+  if (launches_out) *launches_out = s->var_launches[variant];
+  if (bytes_out) *bytes_out = s->var_bytes[variant];
+  if (name_out) *name_out = names[variant];
   return PS_OK;
 }
 
@@ -1404,7 +1631,8 @@ __global__ void ps_noalloc_setup_kernel(NoAllocArgs a) {
     h.parts_per_chunk = 1;
     h.profile = 0;
     h.sparse_off = 0;
-    h._r1 = h._r2 = 0;
+    h.exited = 0;
+    h._r2 = 0;
     *reinterpret_cast<PsTableHdr*>(base) = h;
     *reinterpret_cast<PsTaskDev*>(base + kNaTaskOff) = a.task;     // ticket = 0 inside
     *reinterpret_cast<unsigned int*>(base + kNaStartsOff) = 0;
@@ -1441,8 +1669,10 @@ extern "C" int ps_aggregate_block_noalloc(const ps_job_desc* job, unsigned long 
   if (job->opt == PS_ADAM && !state1) return PS_ERR_BAD_ARG;
   if (nelem > PS_NOALLOC_MAX_ELEMS) return PS_ERR_TOO_LARGE;
   const uintptr_t esz = job->grad_dtype == PS_BF16 ? 2 : 4;
+  // `all` decides between 128-bit and scalar accesses: parameters, state and shards only
+  // (the norm is one double written by a single thread and needs 8-byte alignment, no more)
   uintptr_t all = reinterpret_cast<uintptr_t>(params) | reinterpret_cast<uintptr_t>(state0) |
-                  reinterpret_cast<uintptr_t>(state1) | reinterpret_cast<uintptr_t>(sqnorm_out);
+                  reinterpret_cast<uintptr_t>(state1);
   if ((all & 3u) || (reinterpret_cast<uintptr_t>(sqnorm_out) & 7u)) return PS_ERR_ALIGN;
   for (int w = 0; w < job->num_workers; ++w) {
     if (!shard_ptrs[w]) return PS_ERR_BAD_ARG;
@@ -1495,11 +1725,12 @@ extern "C" int ps_aggregate_block_noalloc(const ps_job_desc* job, unsigned long 
 
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   unsigned char* sc = nd.scratch;
+  cudaGetLastError();   // an error left behind by unrelated earlier work is not this call's
   ps_noalloc_setup_kernel<<<1, PS_MAX_WORKERS, 0, stream>>>(a);
   const int grid = (int)std::min<unsigned long long>(a.task.nchunks, (unsigned long long)nd.num_sms * 3ull);
   ps_aggregate_ldg_kernel<<<grid, kThreads, 0, stream>>>(sc, reinterpret_cast<const PsJobDev*>(sc + kNaJobOff),
                                                          reinterpret_cast<PsStat*>(sc + kNaStatOff),
-                                                         reinterpret_cast<double*>(sc + kNaPartOff));
+                                                         reinterpret_cast<double*>(sc + kNaPartOff), nullptr, 0ull);
   if (sqnorm_out) ps_noalloc_finish_kernel<<<1, 1, 0, stream>>>(sqnorm_out);
   return cudaGetLastError() == cudaSuccess ? PS_OK : PS_ERR_CUDA;
 }

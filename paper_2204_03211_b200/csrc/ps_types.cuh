@@ -56,7 +56,8 @@ struct __align__(16) PsTableHdr {      // 48 bytes at the start of the table
   unsigned int parts_per_chunk;        // partial sums each chunk publishes (1 per CTA or 1 per consumer warp)
   unsigned int profile;                // 1: record per-task device time (direct-load kernel)
   unsigned int sparse_off;             // byte offset of the PsSparseDev array (row-sparse shards)
-  unsigned int _r1, _r2;
+  unsigned int exited;                 // CTAs that have left the launch (uploaded as 0)
+  unsigned int _r2;
 };
 
 // One worker's shard of a row-sparse task: the sorted ids of the rows it holds

@@ -200,6 +200,76 @@ def test_arena_accounting_and_exhaustion():
     assert s.arena_info(0)[0] == 3 * 4096 + 3 * 320_000
 
 
+def test_unaligned_dense_shard_cannot_share_a_block_with_row_sparse_pushes():
+    """A block that holds row-sparse pushes is streamed row by row with 128-bit
+    loads from EVERY shard; a dense shard that is only element-aligned would
+    fault there, so whichever of the two pushes comes second is refused on the
+    host, before anything can be launched."""
+    s = _svc()
+    j = s.register_job(num_workers=3)
+    s.register_block(j, 0, 64)           # 4 rows of 16
+    s.register_block(j, 1, 64)
+    # dense (4-byte aligned only) first, row-sparse second
+    s.push(j, 0, 0, 4096 + 4)
+    assert _status(s.push_rows, j, 0, 1, 8192, 1, 16, 12288) == B.PS_ERR_ALIGN
+    s.push(j, 0, 1, 8192)                # worker 1 can still push dense
+    s.push(j, 0, 2, 12288)
+    assert [c.vector_path for c in s.plan([(j, 0)])] == [0]      # all-dense block: scalar path, allowed
+    # row-sparse first, unaligned dense second
+    s.push_rows(j, 1, 0, 8192, 1, 16, 12288)
+    assert _status(s.push, j, 1, 1, 4096 + 4) == B.PS_ERR_ALIGN
+    assert _status(s.push, j, 1, 1, 4096 + 8) == B.PS_ERR_ALIGN
+    s.push(j, 1, 1, 4096 + 16)           # 16-byte aligned dense shard is fine
+    jobs = np.array([j], np.int32)
+    assert _status(s.push_batch, jobs, np.array([1], np.int32), np.array([2], np.int32),
+                   np.array([4096 + 4], np.uint64)) == B.PS_ERR_ALIGN
+    s.push(j, 1, 2, 16384)
+    assert len(s.plan([(j, 1)])) >= 1
+    # nothing was launched: a planning-only service cannot launch
+    assert s.launch_info()["launches"] == 0
+
+
+def test_round_is_all_or_nothing_and_validates_flags():
+    s = _svc()
+    j = s.register_job(num_workers=2)
+    s.register_block(j, 0, 64)
+    s.register_block(j, 1, 64)
+    jobs = np.array([j, j], np.int32)
+    blocks = np.array([0, 0], np.int32)
+    workers = np.array([0, 1], np.int32)
+    ptrs = np.array([4096, 8192], np.uint64)
+    assert _status(s.round, jobs, blocks, workers, ptrs, [(j, 0)], 2) == B.PS_ERR_BAD_ARG       # unknown flag
+    assert _status(s.plan, [(j, 0)]) == B.PS_ERR_NOT_READY                                      # nothing was pushed
+    # block 1 is listed but has no pushes: the round is refused and block 0's pushes are taken back
+    assert _status(s.round, jobs, blocks, workers, ptrs, [(j, 0), (j, 1)]) == B.PS_ERR_NOT_READY
+    assert _status(s.plan, [(j, 0)]) == B.PS_ERR_NOT_READY
+    # complete round on a planning-only service: validation passes, then the compute step refuses
+    assert _status(s.round, jobs, blocks, workers, ptrs, [(j, 0)], B.PS_ROUND_INPUTS_COMPLETE) == B.PS_ERR_NO_DEVICE
+    assert _status(s.plan, [(j, 0)]) == B.PS_ERR_NOT_READY                                      # and rolls back too
+    s.push_batch(jobs, blocks, workers, ptrs)
+    assert len(s.plan([(j, 0)])) == 1
+
+
+def test_block_table_stays_bounded_when_blocks_come_and_go():
+    """Migration between services registers a block on the new owner and
+    unregisters it on the old one; a planner that moves blocks back and forth
+    must not grow the registry."""
+    s = _svc(ctxs=1, arena=1 << 24)
+    j = s.register_job(num_workers=1, opt=B.PS_ADAM)
+    s.register_block(j, 0, 1000)
+    base = s.registry_info()
+    assert base == dict(jobs=1, blocks=1, block_entries=1)
+    for k in range(10_000):
+        s.register_block(j, 1 + (k % 7), 500 + k % 11)
+        s.unregister_block(j, 1 + (k % 7))
+    info = s.registry_info()
+    assert info["blocks"] == 1 and info["block_entries"] <= 2
+    assert s.arena_info(0)[0] == 3 * 4096            # only block 0's ranges remain
+    s.register_block(j, 3, 2000)
+    s.push(j, 3, 0, 4096)
+    assert sum(c.elem_count for c in s.plan([(j, 3)])) == 2000 and s.block_stats(j, 3) == (0.0, 0)
+
+
 def test_plain_c99_client_compiles_against_the_header_and_runs(tmp_path):
     """The boundary is C: a C99 program built with gcc -pedantic against
     include/ps_b200.h links the library and exercises registration, push
