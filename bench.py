@@ -64,53 +64,91 @@ def measured_peak():
 # ------------------------------------------------------------------ clocks
 
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    """Samples nvidia-smi every 50 ms from before the warm-up until the timed
+    region ends.  clocks.sm / clocks.max.sm are parsed on their own; the
+    throttle-reason fields are optional (a driver that does not know one of
+    them falls back to a query of the two clock fields only)."""
+    FULL = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+            "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+            "clocks_event_reasons.sw_power_cap")
+    BASIC = "clocks.sm,clocks.max.sm"
+    REASONS = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
 
     def __init__(self, index: int):
-        self.index, self.proc, self.path = index, None, None
+        self.index, self.proc, self.path, self.fields, self.note = index, None, None, self.FULL, None
+        self.marks = []
+
+    def _spawn(self, fields):
+        fd, self.path = tempfile.mkstemp(suffix=".csv")
+        os.close(fd)
+        self.fields = fields
+        self.proc = subprocess.Popen(
+            ["nvidia-smi", "-i", str(self.index), "--query-gpu=timestamp," + fields,
+             "--format=csv,noheader,nounits", "-lms", "50"],
+            stdout=open(self.path, "w"), stderr=subprocess.STDOUT)
 
     def start(self):
         try:
-            fd, self.path = tempfile.mkstemp(suffix=".csv")
-            os.close(fd)
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "50"],
-                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            self._spawn(self.FULL)
+            time.sleep(0.25)
+            if self.proc.poll() is not None:           # refused the query: ask for the clocks alone
+                self.note = "full query refused: " + open(self.path).read().strip()[:120]
+                self._spawn(self.BASIC)
+        except Exception as e:                         # noqa: BLE001
+            self.proc, self.note = None, "nvidia-smi could not be started: %r" % (e,)
+
+    def mark(self):
+        """Remembers 'now' (the sampler's own clock: lines written so far)."""
+        try:
+            with open(self.path) as f:
+                self.marks.append(sum(1 for _ in f))
         except Exception:
-            self.proc = None
+            self.marks.append(0)
 
     def stop(self) -> dict:
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "samples_timed_region": 0}
         if not self.proc:
+            out["why_no_samples"] = self.note or "sampler not started"
             return out
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        rows, bad = [], 0
         try:
             for line in open(self.path):
                 f = [x.strip() for x in line.split(",")]
-                if len(f) < 7:
-                    continue
                 try:
-                    sm.append(float(f[0]))
-                    mx.append(float(f[1]))
-                except ValueError:
-                    continue
-                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                    rows.append((float(f[1]), float(f[2]), f[3:]))
+                except (ValueError, IndexError):
+                    bad += 1
+                    rows.append(None)
+            os.unlink(self.path)
+        except Exception as e:                         # noqa: BLE001
+            out["why_no_samples"] = "cannot read the sampler's output: %r" % (e,)
+            return out
+        first = self.marks[0] if self.marks else 0
+        timed = [r for r in rows[first:] if r]
+        every = [r for r in rows if r]
+        use = timed if timed else every
+        if not use:
+            out["why_no_samples"] = (self.note or "") + " no parsable line among %d (%d unparsable)" % (len(rows), bad)
+            return out
+        # under load = the upper half of the samples of the timed region (the lower half may hold the
+        # gaps between blocks of steps)
+        sm = sorted(r[0] for r in use)
+        upper = sm[len(sm) // 2:]
+        reasons = set()
+        if self.fields == self.FULL:
+            for r in use:
+                for name, v in zip(self.REASONS, r[2][1:5]):
                     if v.lower().startswith("active"):
                         reasons.add(name)
-            os.unlink(self.path)
-        except Exception:
-            pass
-        if sm:
-            # under load = the upper half of the samples (the sampler also sees set-up and idle gaps)
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        out.update(sm_mhz=statistics.median(upper), sm_max_mhz=max(r[1] for r in use), reasons=sorted(reasons),
+                   samples=len(every), samples_timed_region=len(timed), sm_mhz_min=sm[0])
+        if self.note:
+            out["note"] = self.note
         return out
 
 
@@ -120,7 +158,8 @@ class Workload:
     """The service, the device-resident gradients and the per-round call
     arguments of one workload, prepared outside any timed region."""
 
-    def __init__(self, cfg: configs.Config, device: int, ticks: int, n_schedules: int, sparse: bool = False):
+    def __init__(self, cfg: configs.Config, device: int, ticks: int, n_schedules: int, sparse: bool = False,
+                 prepared: bool = True):
         from paper_2204_03211_b200 import binding as B
         self.B, self.cfg, self.device = B, cfg, device
         dev = torch.device("cuda", device)
@@ -189,23 +228,35 @@ class Workload:
         # the gradient slabs are written once, before any timed region: every push is of a
         # buffer that is already complete in memory
         self.round_flags = B.PS_ROUND_INPUTS_COMPLETE
+        # the rounds recur every len(schedules) steps with the same buffers: prepared once
+        self.prepared = prepared
+        for rounds in self.schedules:
+            for r in rounds:
+                r["rid"] = None
+                if prepared and r["rows"] is None:
+                    r["rid"] = self.svc.round_prepare(r["jobs"], r["blocks"], r["workers"], r["ptrs"], r["tasks"],
+                                                      self.round_flags)
         self.params_per_step = cfg.num_params
         self.bytes_per_step = cfg.bytes_per_round() - self.sparse_saved
 
     def step(self, k: int, stream) -> int:
-        """Push, aggregate, pull — device-resident gradients.  Returns launches."""
+        """Push, aggregate, pull — device-resident gradients.  Returns the number of rounds."""
         # The C entry points are called with arguments marshalled once, outside
         # the timed region (array addresses as integers): one C-ABI call per round
-        # (ps_round = push, aggregate, pull), plus one for row-sparse pushes if any.
+        # (ps_round_run = push, aggregate, pull of a prepared round; ps_round with the
+        # full argument lists otherwise), plus one for row-sparse pushes if any.
         lib, h, sp = self.lib, self.svc.handle, int(stream.cuda_stream)
         rounds = self.schedules[k % len(self.schedules)]
         flags = self.round_flags
         for r in rounds:
             rc = 0
-            if r["rows"] is not None:
-                rc = lib.ps_push_rows_batch(h, *r["c_rows"])
-            if rc == 0:
-                rc = lib.ps_round(h, *r["c_round"], flags, sp, r["c_pulled"])
+            if r["rid"] is not None:
+                rc = lib.ps_round_run(h, r["rid"], sp, r["c_pulled"])
+            else:
+                if r["rows"] is not None:
+                    rc = lib.ps_push_rows_batch(h, *r["c_rows"])
+                if rc == 0:
+                    rc = lib.ps_round(h, *r["c_round"], flags, sp, r["c_pulled"])
             if rc:
                 raise self.B.PsError(rc, "bench step")
         if self.overlap:
@@ -328,25 +379,43 @@ def whole_job_value(units_per_rank_per_step: int, world: int, steps: int, ms: fl
 
 def timed(fn, steps: int, stream, dist_on: bool, device):
     """Times `steps` calls of fn(k, stream) with CUDA events on `stream`,
-    bracketed by barrier + synchronize; returns (ms max over ranks, launches)."""
+    bracketed by barrier + synchronize; returns (ms max over ranks, rounds, host ms)."""
     import torch.distributed as dist
     torch.cuda.synchronize(device)
     if dist_on:
         dist.barrier()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches = 0
+    rounds = 0
     host0 = time.perf_counter()
     with torch.cuda.stream(stream):
         t0.record(stream)
         for k in range(steps):
-            launches += fn(k, stream)
+            rounds += fn(k, stream)
         t1.record(stream)
     host_ms = (time.perf_counter() - host0) * 1e3
     torch.cuda.synchronize(device)
     if dist_on:
         dist.barrier()
     ms = max_over_ranks(t0.elapsed_time(t1), device)
-    return ms, launches, host_ms
+    return ms, rounds, host_ms
+
+
+def timed_blocks(fn, steps: int, stream, dist_on: bool, device, min_seconds: float, max_blocks: int):
+    """The timed region: blocks of exactly `steps` steps, each bracketed as in
+    timed(), repeated until `min_seconds` of device time have been measured
+    (every rank repeats the same number of times: the count is derived from
+    the first block's max-over-ranks time).  Returns the blocks' times (ms),
+    rounds and host ms."""
+    ms, rounds, host = timed(fn, steps, stream, dist_on, device)
+    blocks, n_rounds, host_ms = [ms], rounds, [host]
+    want = int(min(max_blocks, max(1, -(-min_seconds * 1e3 // max(ms, 1e-3)))))
+    for i in range(1, want):
+        base = i * steps
+        ms, rounds, host = timed(lambda k, st: fn(base + k, st), steps, stream, dist_on, device)
+        blocks.append(ms)
+        host_ms.append(host)
+        n_rounds += rounds
+    return blocks, n_rounds, host_ms
 
 
 # ------------------------------------------------------------------ CPU oracle arm
@@ -422,7 +491,7 @@ def sharded_main(args, cfg, config, rank, local_rank, world, device):
     from paper_2204_03211_b200 import binding as B
     wl.sh.svc.set_option(B.PS_OPT_OVERLAP, int(not args.in_stream))
     wl.fill(0, device)
-    n_sched = max(1, min(args.warmup + args.steps, 8))
+    n_sched = max(1, min(args.warmup, 8))      # every schedule runs once before the timed region
     schedules = [configs.rounds_for(cfg, it, args.ticks) for it in range(n_sched)]
     stream = torch.cuda.Stream(device)
 
@@ -466,22 +535,69 @@ def sharded_main(args, cfg, config, rank, local_rank, world, device):
 
 # ------------------------------------------------------------------ main
 
+def describe(cfg, args) -> dict:
+    """The `config` object of the JSON line: both arms print exactly this."""
+    return {"workload": "%s: %d packed jobs, %d params, %d blocks, W=%s, %s arrival in <=%d rounds/step" % (
+        cfg.name, len(cfg.jobs), cfg.num_params, sum(len(j.blocks) for j in cfg.jobs),
+        sorted({j.num_workers for j in cfg.jobs}), cfg.arrival, args.ticks),
+        "l2": "inputs (%.1f GB/step) exceed L2; no flush" % (cfg.bytes_per_round() / 1e9)
+              if cfg.bytes_per_round() > 4 * 126e6 else
+              "inputs (%.1f MB/step) fit the L2: launch-bound, not an HBM figure" % (cfg.bytes_per_round() / 1e6),
+        "launch_mode": "in-stream" if args.in_stream else "overlapped, one ps_join per step"}
+
+
+def cpu_baseline_all(min_seconds: float):
+    """Oracle throughput on a bounded sample of each of the five configurations."""
+    out = {}
+    for name in sorted(configs.CONFIGS):
+        c = configs.CONFIGS[name]()
+        full_bpp = c.bytes_per_round() / c.num_params
+        # bounded: every job keeps a prefix of its blocks, so that the host generates and the oracle
+        # reads about 1.5 GB per configuration
+        models = len({j.model for j in c.jobs})
+        for job in c.jobs:
+            keep, used = [], 0
+            for b in job.blocks:
+                if keep and (used + b.nelem) * job.bytes_per_elem() > 1.5e9 / models:
+                    break
+                keep.append(b)
+                used += b.nelem
+            job.blocks = keep
+        items, params, desc = oracle_sample(c, None, max_bytes=3e9)
+        v, used, passes, el = time_oracle(items, params, min_seconds, 50)
+        out[name] = {"value": v, "unit": UNIT, "cores": used, "sample": "%s, %d passes in %.1f s" % (desc, passes, el),
+                     "sample_bytes_per_param": sample_bytes_per_param(c, items, params),
+                     "workload_bytes_per_param": full_bpp}
+        del items
+    return out
+
+
+def sample_bytes_per_param(cfg, items, params) -> float:
+    total = 0
+    for (hp, step, shards, p, s0, s1) in items:
+        total += sum(g.nbytes for g in shards) + 2 * p.nbytes + 2 * s0.nbytes + (2 * s1.nbytes if s1 is not None else 0)
+    return total / max(params, 1)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C4", choices=sorted(configs.CONFIGS))
     ap.add_argument("--ticks", type=int, default=16, help="rounds per iteration window of the arrival schedule")
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--min-seconds", type=float, default=2.0,
+                    help="the block of --steps steps is repeated until this much device time has been measured")
+    ap.add_argument("--max-blocks", type=int, default=400, help="upper bound on those repetitions")
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--e2e-mode", default="mapped", choices=["staged", "mapped"],
-                    help="staged: only the e2e leg whose shards ps_push_host copies into device staging; mapped: "
+                    help="staged: only the e2e leg whose shards are copied into device staging; mapped: "
                          "also a second leg (e2e_mapped) whose pinned shards are pushed as they are and read by "
                          "the kernel over PCIe")
     ap.add_argument("--host-pool-gb", type=float, default=8.0)
     ap.add_argument("--jobs", default="", help="comma-separated subset of the workload's jobs (profiling a small case)")
-    ap.add_argument("--max-blocks", type=int, default=0, help="keep only the first N blocks of every job")
+    ap.add_argument("--first-blocks", type=int, default=0, help="keep only the first N blocks of every job")
     ap.add_argument("--chunk-elems", type=int, default=0, help="PS_OPT_CHUNK_ELEMS (0 = automatic)")
     ap.add_argument("--kernel", type=int, default=0, help="PS_OPT_KERNEL (0 = automatic, 1 = direct loads, 2 = bulk-copy ring)")
     ap.add_argument("--sparse-transport", action="store_true",
@@ -490,14 +606,21 @@ def main():
     ap.add_argument("--in-stream", action="store_true",
                     help="enqueue every launch on the caller's stream (PS_OPT_OVERLAP = 0) instead of letting "
                          "the launches of a step overlap on the service's streams and joining once per step")
+    ap.add_argument("--no-batch", action="store_true", help="PS_OPT_BATCH = 0: one launch per round, never packed")
+    ap.add_argument("--streams", type=int, default=0, help="PS_OPT_WORK_STREAMS (0 = the library's default)")
+    ap.add_argument("--unprepared", action="store_true",
+                    help="call ps_round with the full argument lists every round instead of ps_round_run on "
+                         "rounds prepared once")
+    ap.add_argument("--no-pdl", action="store_true", help="PS_OPT_PDL = 0: plain launches for small rounds")
     ap.add_argument("--shard-blocks", action="store_true",
                     help="with --gpus N > 1: ONE workload whose blocks are owned by the N ranks (strong scaling; "
                          "shards are read in place from the worker ranks' exported buffers) instead of N replicas")
     ap.add_argument("--dist-backend", default="nccl", choices=["nccl", "gloo"],
                     help="process-group backend for the barriers and the max over ranks")
-    ap.add_argument("--no-pdl", action="store_true", help="PS_OPT_PDL = 0: plain launches for small rounds")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cpu-baseline-all", action="store_true",
+                    help="skip timing the oracle on a bounded sample of each of the five configurations")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -508,21 +631,20 @@ def main():
     if args.jobs:
         cfg.jobs = [cfg.jobs[int(x)] for x in args.jobs.split(",")]
         cfg.name += "[jobs %s]" % args.jobs
-    if args.max_blocks:
+    if args.first_blocks:
         for job in cfg.jobs:
-            job.blocks = job.blocks[:args.max_blocks]
-        cfg.name += "[first %d blocks]" % args.max_blocks
-    config = {"workload": "%s: %d packed jobs, %d params, %d blocks, W=%s, %s arrival in <=%d rounds/step" % (
-        cfg.name, len(cfg.jobs), cfg.num_params, sum(len(j.blocks) for j in cfg.jobs),
-        sorted({j.num_workers for j in cfg.jobs}), cfg.arrival, args.ticks),
-        "l2": "inputs (%.1f GB/step) exceed L2; no flush" % (cfg.bytes_per_round() / 1e9)}
+            job.blocks = job.blocks[:args.first_blocks]
+        cfg.name += "[first %d blocks]" % args.first_blocks
+    config = describe(cfg, args)
 
     if args.impl == "reference":
+        # The only reference this path has is the CPU oracle: timed as it stands on the host cores,
+        # each step one aggregate of a bounded sample of the workload.
         if rank != 0:
             return 0
         items, params, desc = oracle_sample(cfg)
         from oracle import aggregator as A
-        for _ in range(min(args.warmup, 1)):
+        for _ in range(args.warmup):
             A.run_blocks(items, 0)
         t = time.perf_counter()
         used = 1
@@ -532,10 +654,12 @@ def main():
         val = params * args.steps / dt
         print(json.dumps({
             "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": dt / args.steps * 1e3,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic", "config": config,
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": used, "kind": "oracle", "sample": desc},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": used, "kind": "oracle", "sample": desc,
+                             "sample_bytes_per_param": sample_bytes_per_param(cfg, items, params),
+                             "workload_bytes_per_param": cfg.bytes_per_round() / cfg.num_params},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}))
         return 0
@@ -555,35 +679,59 @@ def main():
     if args.shard_blocks and dist_on:
         return sharded_main(args, cfg, config, rank, local_rank, world, device)
 
-    n_sched = max(1, min(args.warmup + args.steps, 8))
-    wl = Workload(cfg, local_rank, args.ticks, n_sched, sparse=args.sparse_transport)
+    # the clocks are sampled from before the warm-up, so that even a short timed region has samples
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+
+    n_sched = max(1, min(args.warmup, 8))      # every schedule runs once before the timed region
+    wl = Workload(cfg, local_rank, args.ticks, n_sched, sparse=args.sparse_transport, prepared=not args.unprepared)
+    B = wl.B
     if args.sparse_transport:
         args.no_e2e = True
         config["transport"] = "row-sparse pushes for embedding tables: %.2f GB of gradient reads avoided per step" % (
             wl.sparse_saved / 1e9)
-    wl.svc.set_option(wl.B.PS_OPT_CHUNK_ELEMS, args.chunk_elems)
-    wl.svc.set_option(wl.B.PS_OPT_KERNEL, args.kernel)
-    wl.svc.set_option(wl.B.PS_OPT_PDL, int(not args.no_pdl))
+    wl.svc.set_option(B.PS_OPT_CHUNK_ELEMS, args.chunk_elems)
+    wl.svc.set_option(B.PS_OPT_KERNEL, args.kernel)
+    wl.svc.set_option(B.PS_OPT_PDL, int(not args.no_pdl))
+    wl.svc.set_option(B.PS_OPT_BATCH, int(not args.no_batch))
+    if args.streams:
+        wl.svc.set_option(B.PS_OPT_WORK_STREAMS, args.streams)
     wl.overlap = not args.in_stream
-    wl.svc.set_option(wl.B.PS_OPT_OVERLAP, int(wl.overlap))
-    config["launch_mode"] = "overlapped, one ps_join per step" if wl.overlap else "in-stream"
+    wl.svc.set_option(B.PS_OPT_OVERLAP, int(wl.overlap))
     stream = torch.cuda.Stream(device)
 
     for k in range(args.warmup):
         wl.step(k, stream)
-    sampler = ClockSampler(local_rank)
+    torch.cuda.synchronize(device)
     if rank == 0:
-        sampler.start()
-    l0 = wl.svc.launch_info()["launches"]
+        sampler.mark()
+    stats0 = wl.svc.launch_stats()
     red_dev = device if args.dist_backend == "nccl" else None      # where the max over ranks is reduced
-    ms, launches, host_ms = timed(lambda k, s: wl.step(args.warmup + k, s), args.steps, stream, dist_on, red_dev)
+    blocks, rounds, host_ms = timed_blocks(lambda k, s: wl.step(args.warmup + k, s), args.steps, stream, dist_on,
+                                           red_dev, args.min_seconds, args.max_blocks)
     clocks = sampler.stop() if rank == 0 else {}
+    stats1 = wl.svc.launch_stats()
     info = wl.svc.launch_info()
-    assert info["launches"] - l0 == launches
+    ms = statistics.median(blocks)                                   # one block of exactly --steps steps
     value = whole_job_value(wl.params_per_step, world, args.steps, ms)
     achieved = wl.bytes_per_step * args.steps / (ms * 1e-3) / 1e9     # per GPU
     peak, peak_kind = measured_peak()
-    per_launch_bytes = wl.bytes_per_step * args.steps / launches
+    # the kernels of the timed region: launches and algorithmic bytes per variant
+    mix = []
+    for v0, v1 in zip(stats0, stats1):
+        n, by = v1["launches"] - v0["launches"], v1["bytes"] - v0["bytes"]
+        if n:
+            mix.append({"kernel": v1["kernel"], "launches": n, "bytes": by})
+    total_bytes = sum(m["bytes"] for m in mix) or 1
+    for m in mix:
+        m["byte_share"] = m["bytes"] / total_bytes
+    dominant = max(mix, key=lambda m: m["bytes"]) if mix else {"kernel": "none", "launches": 0, "bytes": 0}
+    launches = sum(m["launches"] for m in mix)
+    per_launch_bytes = dominant["bytes"] / max(dominant["launches"], 1)
+    # the dominant kernel's average launch duration: the timed region's device time, less nothing —
+    # its launches fill the region (other variants' byte share is printed beside it)
+    dom_ms = sum(blocks) * dominant.get("byte_share", 1.0) / max(dominant["launches"], 1)
     sha = kernel_sha()
     traffic = None
     if NCU_TRAFFIC["kernel_sha"] == sha and NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"]:
@@ -592,43 +740,59 @@ def main():
     e2e = e2e_mapped = None
     if not args.no_e2e:
         wl.prepare_host(int(args.host_pool_gb * (1 << 30)))
+
         def host_leg(host_step, mode):
             host_step(0, stream)        # warm-up (staged: allocates the staging buffers)
             torch.cuda.synchronize(device)
             ems, _, _ = timed(host_step, args.e2e_steps, stream, dist_on, red_dev)
             return {"value": whole_job_value(wl.params_per_step, world, args.e2e_steps, ems), "unit": UNIT,
                     "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "steps": args.e2e_steps,
-                    "ms_per_step": ems / args.e2e_steps, "mode": mode, "host_pool_bytes": wl.pool_bytes}
+                    "ms_per_step": ems / args.e2e_steps, "mode": mode, "host_pool_bytes": wl.pool_bytes,
+                    "h2d_gbs": wl.h2d * args.e2e_steps / (ems * 1e-3) / 1e9}
 
-        # staged: ps_push_host copies every shard from pinned memory into device staging, then the kernel
+        # staged: the round's shards are copied from pinned memory into device staging, then the kernel
         # reads the staging; mapped: the pinned shards themselves are pushed (ps_push) and the kernel
         # reads them over PCIe in place.  Same bytes cross the link every step in both.
-        e2e = host_leg(wl.step_host, "staged: ps_push_host copies, then aggregate")
+        e2e = host_leg(wl.step_host, "staged: host shards copied to device staging, then aggregate")
         if args.e2e_mode == "mapped":
             e2e_mapped = host_leg(wl.step_host_mapped, "mapped: ps_push of pinned host pointers, the kernel reads over PCIe")
 
-    cpu = None
+    cpu = cpu_all = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         items, params, desc = oracle_sample(cfg, wl.slabs)
         v, used, passes, el = time_oracle(items, params, 12.0, 1000)
         cpu = {"value": v, "unit": UNIT, "cores": used, "kind": "oracle",
-               "sample": "%s, %d passes in %.1f s" % (desc, passes, el)}
+               "sample": "%s, %d passes in %.1f s" % (desc, passes, el),
+               "sample_bytes_per_param": sample_bytes_per_param(cfg, items, params),
+               "workload_bytes_per_param": cfg.bytes_per_round() / cfg.num_params}
+        del items
+        if not args.no_cpu_baseline_all:
+            cpu_all = cpu_baseline_all(2.0)
 
     if rank == 0:
+        frac_nominal = achieved / 8000.0
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+            "timed_region": {"blocks": len(blocks), "steps_per_block": args.steps, "ms_per_step": "median block",
+                             "ms_per_step_min": min(blocks) / args.steps, "ms_per_step_max": max(blocks) / args.steps,
+                             "seconds": sum(blocks) / 1e3, "rounds": rounds, "launches": launches},
             "hbm_gbs_algorithmic": achieved,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": traffic, "peak_source": peak_kind + " copy bandwidth",
-                         "frac_of_nominal_8TBs": achieved / 8000.0, "kernel": info["kernel"],
-                         "bytes_per_launch": per_launch_bytes, "kernel_sha": sha,
-                         "note": "duration = event time of the whole timed region / launches "
-                                 "(launches of a step may overlap; table uploads included)"},
-            "cpu_baseline": cpu, "e2e": e2e, "e2e_mapped": e2e_mapped, "gpu_launches": launches,
+                         "frac": achieved / peak, "traffic": traffic,
+                         "peak_source": peak_kind + " copy bandwidth (half reads, half writes; this path mostly "
+                                                    "reads, so the ratio can exceed 1)",
+                         "frac_of_nominal_8TBs": frac_nominal, "kernel": dominant["kernel"],
+                         "kernel_share": dominant.get("byte_share"), "kernels": mix,
+                         "bytes_per_launch": per_launch_bytes, "launch_ms": dom_ms, "kernel_sha": sha,
+                         "note": "achieved = algorithmic bytes of a block of steps / its event time (launches of a "
+                                 "step overlap and pack; table uploads included); launch_ms = the dominant kernel's "
+                                 "share of that time / its launches"},
+            "cpu_baseline": cpu, "cpu_baseline_all": cpu_all, "e2e": e2e, "e2e_mapped": e2e_mapped,
+            "gpu_launches": launches,
             "launch": {"grid": info["grid"], "block": info["block"]},
-            "host_ms_per_step": host_ms / args.steps, "clocks": clocks,
+            "host_ms_per_step": statistics.median(host_ms) / args.steps, "clocks": clocks,
         }
         print(json.dumps(line))
     wl.svc.close()

@@ -100,6 +100,18 @@ enum {
                               overlaps the tail of the previous launch of the same stream, and the
                               kernel waits for that launch to complete before it touches any data.
                               0: plain launches.  Same results. */
+  PS_OPT_BATCH = 10,       /* 1 (default), effective with PS_OPT_OVERLAP for rounds given with
+                              PS_ROUND_INPUTS_COMPLETE: packing over time.  While at least two launches
+                              of the service are still running, such a round is not launched but held
+                              back and packed into ONE launch with the rounds that follow it; the batch
+                              goes out when the device is about to run dry, when it fills two waves of
+                              CTAs, at ps_join / ps_flush, and before any call that reads or moves the
+                              blocks' state (ps_block_stats, ps_pull_host, ps_migrate_block, a push for a
+                              block that waits in the batch, ...).  An idle device gets every round at
+                              once.  Results are identical; what changes is how many launches carry
+                              them.  0: one launch per round. */
+  PS_OPT_WORK_STREAMS = 9, /* with PS_OPT_OVERLAP: launches rotate over this many service-owned streams
+                              (1..8, default 4) */
   PS_OPT_PROFILE = 5,      /* 1: aggregates record per-task device time (see ps_block_profile);
                               costs a few atomics per chunk; direct-load kernel only; default 0 */
   PS_OPT_KERNEL = 4        /* kernel variant: 0 = automatic (direct loads), 1 = direct loads,
@@ -205,6 +217,11 @@ int ps_aggregate(ps_service* svc, const ps_task* ready, int n_ready, void* strea
  * not joined yet (needed only with PS_OPT_OVERLAP; otherwise a no-op). */
 int ps_join(ps_service* svc, void* stream);
 
+/* Launches whatever PS_OPT_BATCH is holding back, without making any stream
+ * wait (ps_join does both).  A caller that stops issuing rounds calls one of
+ * the two; until then held-back rounds have not started. */
+int ps_flush(ps_service* svc);
+
 /* One round of the service in ONE call — what an Aggregator does when the last
  * worker's gradients of some tensors have arrived (paper Figure 1 and Section 2.1:
  * tensors become ready one layer after another during the backward pass, so a
@@ -258,6 +275,28 @@ int ps_migrate_block(ps_service* svc, int job, int block, int dst_ctx, void* str
  * exactly that case: the overhead of migrating all tensors of a model).
  * Errors: BAD_ARG, DUPLICATE, NOMEM, NO_DEVICE, CUDA. */
 int ps_migrate_blocks(ps_service* svc, const ps_task* tasks, int n, int dst_ctx, void* stream);
+
+/* A round that recurs.  Training is iterative (paper Section 2.2, "Iterative
+ * Training"; Section 3.3.1 builds cyclic execution on it): iteration after
+ * iteration the same tensors become ready in the same groups, pushed from the
+ * same buffers.  ps_round_prepare records one such round — the arguments of
+ * ps_round, copied — and returns a small integer; ps_round_run(round) then does
+ * exactly what ps_round would do with those arguments, but the lists are already
+ * resolved and, when the round's pushes are precisely the W shards of each of
+ * its ready blocks, the packed task table of the previous run is reused with
+ * only the step-dependent fields refreshed.  A run therefore costs the host
+ * little more than the kernel launch.  Anything that could change the table
+ * (a migration, ps_unregister_block, an option) makes the next run resolve and
+ * build again by itself; a round whose block has been unregistered fails with
+ * BAD_ARG.  params_dev_ptrs_out (may be NULL) receives the n_ready parameter
+ * pointers.  ps_round_release forgets a round (its number may be handed out
+ * again).  Errors of ps_round_prepare: BAD_ARG, ALIGN, DUPLICATE (task listed
+ * twice).  Errors of ps_round_run: those of ps_round; all-or-nothing alike. */
+int ps_round_prepare(ps_service* svc, int n_push, const int* jobs, const int* blocks, const int* workers,
+                     const void* const* grad_dev_ptrs, const ps_task* ready, int n_ready, unsigned int flags,
+                     int* round_out);
+int ps_round_run(ps_service* svc, int round, void* stream, const float** params_dev_ptrs_out);
+int ps_round_release(ps_service* svc, int round);
 
 /* Per-block statistics of the last aggregate (paper Section 3.1: profilers feed
  * the manager): squared norm of the aggregated gradient and the step counter.

@@ -28,6 +28,8 @@ PS_OPT_CHUNK_ELEMS, PS_OPT_CTAS_PER_SM, PS_OPT_SORT_TASKS, PS_OPT_KERNEL, PS_OPT
 PS_OPT_OVERLAP = 6
 PS_OPT_INLINE_TABLE = 7
 PS_OPT_PDL = 8
+PS_OPT_WORK_STREAMS = 9
+PS_OPT_BATCH = 10
 PS_ROUND_INPUTS_COMPLETE = 1
 
 
@@ -67,8 +69,13 @@ _SIGNATURES = {
     "ps_push_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
     "ps_aggregate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "ps_join": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "ps_flush": (C.c_int, [C.c_void_p]),
     "ps_round": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                            C.c_uint, C.c_void_p, C.c_void_p]),
+    "ps_round_prepare": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                   C.c_int, C.c_uint, C.POINTER(C.c_int)]),
+    "ps_round_run": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]),
+    "ps_round_release": (C.c_int, [C.c_void_p, C.c_int]),
     "ps_launch_stats": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_ulonglong), C.POINTER(C.c_ulonglong),
                                   C.POINTER(C.c_char_p)]),
     "ps_pull": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p)]),
@@ -256,6 +263,26 @@ def ps_round(svc, jobs, blocks, workers, ptrs, ready, flags: int = 0, stream=Non
     return out
 
 
+def ps_round_prepare(svc, jobs, blocks, workers, ptrs, ready, flags: int = 0) -> int:
+    """Records a recurring round (arguments as for ps_round, copied by the
+    library); returns its number for ps_round_run."""
+    tasks = ready if isinstance(ready, C.Array) else make_tasks(list(ready))
+    n = 0 if jobs is None else len(jobs)
+    out = C.c_int(-1)
+    _check(load().ps_round_prepare(svc, n, _ptr(jobs), _ptr(blocks), _ptr(workers), _ptr(ptrs), tasks, len(tasks),
+                                   flags, C.byref(out)), "ps_round_prepare", svc)
+    return out.value
+
+
+def ps_round_run(svc, round_id: int, stream=None, out=None):
+    _check(load().ps_round_run(svc, round_id, _stream_ptr(stream), _ptr(out)), "ps_round_run", svc)
+    return out
+
+
+def ps_round_release(svc, round_id: int):
+    _check(load().ps_round_release(svc, round_id), "ps_round_release", svc)
+
+
 def ps_launch_stats(svc):
     """[{kernel, launches, bytes}] per kernel variant."""
     res = []
@@ -264,6 +291,10 @@ def ps_launch_stats(svc):
         _check(load().ps_launch_stats(svc, v, C.byref(n), C.byref(b), C.byref(name)), "ps_launch_stats", svc)
         res.append(dict(kernel=(name.value or b"").decode(), launches=n.value, bytes=b.value))
     return res
+
+
+def ps_flush(svc):
+    _check(load().ps_flush(svc), "ps_flush", svc)
 
 
 def ps_pull(svc, job: int, block: int) -> int:
@@ -555,7 +586,7 @@ def _bind(name):
     return method
 
 
-for _n in ("round", "launch_stats", "registry_info", "register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "aggregate", "join", "pull", "pull_batch", "pull_host",
+for _n in ("flush", "round", "round_prepare", "round_run", "round_release", "launch_stats", "registry_info", "register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "aggregate", "join", "pull", "pull_batch", "pull_host",
            "migrate_block", "migrate_blocks", "block_stats", "block_profile", "job_profile", "block_state", "plan", "set_option", "get_option", "arena_info",
            "launch_info", "device_status", "block_export", "block_import", "unregister_block", "arena_export", "block_location"):
     setattr(Service, _n, _bind(_n))

@@ -63,15 +63,12 @@ ps_aggregate_ldg_kernel(unsigned char* __restrict__ table, const PsJobDev* __res
     for (int o = 16; o > 0; o >>= 1) sq += __shfl_down_sync(0xffffffffu, sq, o);
     if (lane == 0) s_red[warp] = sq;
     __syncthreads();
-    if (warp == 0) {
-      double s = 0.0;
-      if (lane == 0) {
-        s = s_red[0];
+    if (tid == 0) {
+      double s = s_red[0];
 #pragma unroll
-        for (int k = 1; k < kThreads / 32; ++k) s += s_red[k];
-        if (profile) profile_chunk(tasks + t, t_begin, global_ns());
-      }
-      publish_part(tasks, t, idx, 1u, s, stats, partials, lane);
+      for (int k = 1; k < kThreads / 32; ++k) s += s_red[k];
+      if (profile) profile_chunk(tasks + t, t_begin, global_ns());
+      publish_one(tasks, t, idx, s, stats, partials);
     }
     buf ^= 1;
   }

@@ -362,6 +362,32 @@ __device__ __forceinline__ void publish_part(PsTaskDev* tasks, unsigned int t, u
   }
 }
 
+// The same for ONE calling thread, which adds the partials in chunk order itself.
+// For the persistent kernel: a task there has at most a few
+// hundred chunks, the other CTAs keep streaming while one thread adds, and keeping
+// the other 31 lanes of the warp out of it keeps the chunk loop's registers free.
+__device__ __forceinline__ void publish_one(PsTaskDev* tasks, unsigned int t, unsigned int slot, double s,
+                                            PsStat* stats, double* partials) {
+  const PsTaskDev* T = tasks + t;
+  const unsigned int n = T->nchunks;
+  const double* mine = partials + T->first_chunk;
+  __stcg(partials + slot, s);
+  __threadfence();
+  if (atomicAdd(&tasks[t].ticket, 1u) != n - 1) return;
+  __threadfence();
+  double tot = 0.0;
+  for (unsigned int k = 0; k < n; ++k) tot += __ldcg(mine + k);     // (unrolled, it spilled in the chunk loop: -3 %)
+  PsStat st;
+  st.sqnorm = tot;
+  st.step = T->step;
+  st.busy_ns = __ldcg(&T->busy_ns);
+  const unsigned long long tf = __ldcg(&T->t_first);
+  st.t_first = (tf == ~0ull) ? 0ull : tf;
+  st.t_last = __ldcg(&T->t_last);
+  st._r0 = 0;
+  stats[T->stat_idx] = st;
+}
+
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));

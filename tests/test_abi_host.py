@@ -250,6 +250,42 @@ def test_round_is_all_or_nothing_and_validates_flags():
     assert len(s.plan([(j, 0)])) == 1
 
 
+def test_prepared_round_has_the_semantics_of_ps_round():
+    s = _svc()
+    j = s.register_job(num_workers=2)
+    s.register_block(j, 0, 64)
+    s.register_block(j, 1, 64)
+    jobs = np.array([j, j], np.int32)
+    blocks = np.array([0, 0], np.int32)
+    workers = np.array([0, 1], np.int32)
+    ptrs = np.array([4096, 8192], np.uint64)
+    assert _status(s.round_prepare, jobs, blocks, workers, ptrs, [(j, 0)], 4) == B.PS_ERR_BAD_ARG            # flag
+    assert _status(s.round_prepare, jobs, np.array([0, 7], np.int32), workers, ptrs, [(j, 0)]) == B.PS_ERR_BAD_ARG
+    assert _status(s.round_prepare, jobs, blocks, np.array([0, 2], np.int32), ptrs, [(j, 0)]) == B.PS_ERR_BAD_ARG
+    assert _status(s.round_prepare, jobs, blocks, workers, np.array([4096, 8194], np.uint64), [(j, 0)]) == B.PS_ERR_ALIGN
+    assert _status(s.round_prepare, jobs, blocks, workers, ptrs, [(j, 0), (j, 0)]) == B.PS_ERR_DUPLICATE
+    r = s.round_prepare(jobs, blocks, workers, ptrs, [(j, 0)], B.PS_ROUND_INPUTS_COMPLETE)
+    r2 = s.round_prepare(jobs, blocks, workers, ptrs, [(j, 0), (j, 1)])     # block 1 never gets its pushes
+    assert (r, r2) == (0, 1)
+    assert _status(s.round_run, r2) == B.PS_ERR_NOT_READY
+    assert _status(s.plan, [(j, 0)]) == B.PS_ERR_NOT_READY                  # its pushes were taken back
+    assert _status(s.round_run, r) == B.PS_ERR_NO_DEVICE                    # valid round, planning-only service
+    assert _status(s.plan, [(j, 0)]) == B.PS_ERR_NOT_READY
+    s.push(j, 0, 1, 8192)
+    assert _status(s.round_run, r) == B.PS_ERR_DUPLICATE                    # worker 1 has pushed already
+    s.push(j, 0, 0, 4096)
+    assert len(s.plan([(j, 0)])) == 1                                       # the manual pushes are still there
+    assert _status(s.round_run, 5) == B.PS_ERR_BAD_ARG
+    s.round_release(r2)
+    assert _status(s.round_run, r2) == B.PS_ERR_BAD_ARG
+    assert s.round_prepare(jobs, blocks, workers, ptrs, [(j, 0)]) == r2      # the number is handed out again
+    # a round whose block disappears fails cleanly; one that is registered again resolves again
+    s.unregister_block(j, 0)
+    assert _status(s.round_run, r) == B.PS_ERR_BAD_ARG
+    s.register_block(j, 0, 128)
+    assert _status(s.round_run, r) == B.PS_ERR_NO_DEVICE
+
+
 def test_block_table_stays_bounded_when_blocks_come_and_go():
     """Migration between services registers a block on the new owner and
     unregisters it on the old one; a planner that moves blocks back and forth
