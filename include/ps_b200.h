@@ -105,7 +105,8 @@ enum {
                               of the service are still running, such a round is not launched but held
                               back and packed into ONE launch with the rounds that follow it; the batch
                               goes out when the device is about to run dry, when it fills two waves of
-                              CTAs, at ps_join / ps_flush, and before any call that reads or moves the
+                              CTAs while fewer than six launches are running, when it fills sixteen
+                              waves, at ps_join / ps_flush, and before any call that reads or moves the
                               blocks' state (ps_block_stats, ps_pull_host, ps_migrate_block, a push for a
                               block that waits in the batch, ...).  An idle device gets every round at
                               once.  Results are identical; what changes is how many launches carry

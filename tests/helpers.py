@@ -263,3 +263,100 @@ class SampledPair:
                 assert abs(sq - rsq) <= sq_rtol * abs(rsq) + 1e-300, tag + " sqnorm of block %d" % bid
             for b in job.blocks[:: max(1, len(job.blocks) // 16)]:
                 assert self.svc.block_stats(j, b.block)[1] == expect_step
+
+
+class FullPair:
+    """Full-size configurations compared IN FULL: the CUDA service and the
+    oracle both hold every block; every iteration the gradients are generated
+    on the GPU, the service aggregates them round by round, and the oracle
+    receives a host copy of exactly those bits, job by job (the largest slab is
+    a few GB), and follows every element of every block.  compare() then checks
+    every element of parameters and optimizer state bit for bit, every block's
+    step counter, context and gradient norm.  Launch configuration = what
+    bench.py times (overlapped launches, rounds given with their inputs
+    complete, packing over time)."""
+
+    def __init__(self, cfg: configs.Config, device: int = 0, overlap: int = 1):
+        self.cfg = cfg
+        self.dev = torch.device("cuda", device)
+        arena = sum(3 * (4 * b.nelem + 256) for j in cfg.jobs for b in j.blocks) + (64 << 20)
+        self.svc = B.Service(device, cfg.num_contexts, arena)
+        self.svc.set_option(B.PS_OPT_OVERLAP, overlap)
+        self.ora = A.OracleAggregator(cfg.num_contexts, 0)
+        self.ctx = {}
+        for j, job in enumerate(cfg.jobs):
+            assert self.svc.register_job(**job.hparams()) == j == self.ora.register_job(oracle_hp(job))
+            p0 = generate.init_params(cfg, j, self.dev)
+            h0 = p0.cpu().numpy()
+            for b in job.blocks:
+                c = configs.initial_context(cfg, j, b.block)
+                self.ctx[(j, b.block)] = c
+                self.svc.register_block(j, b.block, b.nelem, c, p0[b.job_offset:b.job_offset + b.nelem])
+                self.ora.register_block(j, b.block, b.nelem, c, h0[b.job_offset:b.job_offset + b.nelem])
+            del p0, h0
+        self.slabs = [None] * len(cfg.jobs)
+        self.stream = torch.cuda.Stream(self.dev)
+
+    def close(self):
+        self.svc.close()
+
+    def iteration(self, it: int, rounds):
+        cfg = self.cfg
+        for j in range(len(cfg.jobs)):
+            self.slabs[j] = generate.grad_slab(cfg, j, it, self.dev, out=self.slabs[j])
+        torch.cuda.synchronize(self.dev)          # the gradients are complete before they are pushed
+        for ready in rounds:
+            jobs, blocks, workers, ptrs = [], [], [], []
+            for (j, b) in ready:
+                job = cfg.jobs[j]
+                for w in range(job.num_workers):
+                    jobs.append(j); blocks.append(b); workers.append(w)
+                    ptrs.append(generate.shard_ptr(self.slabs[j], w, job.blocks[b].job_offset))
+            self.svc.round(np.array(jobs, np.int32), np.array(blocks, np.int32), np.array(workers, np.int32),
+                           np.array(ptrs, np.uint64), ready, B.PS_ROUND_INPUTS_COMPLETE, self.stream)
+        self.svc.join(self.stream)
+        # the oracle: the same bits, every block, one job's slab on the host at a time
+        for j, job in enumerate(cfg.jobs):
+            host = to_np(self.slabs[j])
+            ready = []
+            for b in job.blocks:
+                for w in range(job.num_workers):
+                    self.ora.push(j, b.block, w, host[w, b.job_offset:b.job_offset + b.nelem])
+                ready.append((j, b.block))
+            self.ora.aggregate(ready)
+            del host
+        self.stream.synchronize()
+
+    def migrate(self, plan, stream=None):
+        """Moves every listed block to the next context: one batched call per destination."""
+        by_dst = {}
+        for (j, b) in plan:
+            dst = (self.ctx[(j, b)] + 1) % self.cfg.num_contexts
+            by_dst.setdefault(dst, []).append((j, b))
+            self.ctx[(j, b)] = dst
+            self.ora.migrate_block(j, b, dst)
+        for dst, tasks in by_dst.items():
+            self.svc.migrate_blocks(tasks, dst, stream)
+
+    def compare(self, expect_step: int, sq_rtol: float = 1e-5):
+        assert self.svc.device_status() == 0
+        torch.cuda.synchronize(self.dev)
+        elems = 0
+        for j, job in enumerate(self.cfg.jobs):
+            for b in job.blocks:
+                tag = "%s job %d block %d" % (self.cfg.name, j, b.block)
+                s0, s1, ctx = self.svc.block_state(j, b.block)
+                assert ctx == self.ctx[(j, b.block)] == self.ora.blocks[(j, b.block)].ctx, tag + " context"
+                ra, rv = self.ora.state(j, b.block)
+                got = self.svc.view(self.svc.pull(j, b.block), b.nelem).cpu().numpy()
+                assert np.array_equal(got, self.ora.pull(j, b.block)), tag + " params not bit-identical"
+                assert np.array_equal(self.svc.view(s0, b.nelem).cpu().numpy(), ra), tag + " state0 not bit-identical"
+                if rv is not None:
+                    assert np.array_equal(self.svc.view(s1, b.nelem).cpu().numpy(), rv), tag + " state1 not bit-identical"
+                sq, step = self.svc.block_stats(j, b.block)
+                rsq, rstep = self.ora.block_stats(j, b.block)
+                assert step == rstep == expect_step, tag + " step"
+                assert abs(sq - rsq) <= sq_rtol * abs(rsq) + 1e-300, tag + " sqnorm %r vs %r" % (sq, rsq)
+                elems += b.nelem
+        assert elems == self.cfg.num_params
+        return elems

@@ -1,17 +1,21 @@
-"""The five benchmark configurations at full size, CUDA path vs CPU oracle.
+"""The five benchmark configurations at full size, CUDA path vs CPU oracle,
+every element of every block.
 
-C1 and C2 are compared in full (every element of every block); C3, C4 and C5
-are too large for the oracle to follow whole within seconds, so every block is
-checked at a seeded sample of positions (edges, chunk boundaries, interior)
-plus a few whole blocks per job — the update is element-wise, so the oracle's
-values at those positions are exact.  Launch configuration = the library's
-defaults, which is what bench.py times.
+The oracle follows all iterations in full: each iteration's gradients are
+generated on the GPU and handed to it as host copies, one job's slab at a time;
+after the first and the last iteration (C5: also after the first one that
+follows the migration) every element of parameters and optimizer state is
+compared bit for bit, and every block's step, context and gradient norm.
+Launch configuration = the one bench.py times: overlapped launches, rounds
+given with their inputs complete, packing over time.  C2's 50-iteration
+layer-by-layer replay additionally runs with the sampled checker, as a second,
+independent path through the comparison code.
 """
 import numpy as np
 import pytest
 import torch
 
-from helpers import Pair, SampledPair
+from helpers import FullPair, Pair, SampledPair
 from workload import configs
 
 pytestmark = pytest.mark.gpu
@@ -44,60 +48,65 @@ def test_c2_all_blocks_in_full_three_iterations_all_at_once():
         pair.close()
 
 
-def test_c3_vgg16_shaped_20_iterations():
+def test_c2_layer_by_layer_in_full_every_element():
+    cfg = configs.c2()
+    pair = FullPair(cfg)
+    try:
+        rounds = configs.rounds_for(cfg, 0)
+        for it in range(cfg.iterations):
+            pair.iteration(it, rounds)
+            if it in (0, cfg.iterations - 1):
+                assert pair.compare(it + 1) == cfg.num_params
+    finally:
+        pair.close()
+
+
+def test_c3_vgg16_shaped_20_iterations_every_element():
     cfg = configs.c3()
-    pair = SampledPair(cfg, per_block=256, full_per_job=4)
+    pair = FullPair(cfg)
     try:
         rounds = configs.rounds_all(cfg)
         for it in range(cfg.iterations):
             pair.iteration(it, rounds)
             if it in (0, cfg.iterations - 1):
-                pair.compare(it + 1)
+                assert pair.compare(it + 1) == cfg.num_params
     finally:
         pair.close()
 
 
 @pytest.mark.parametrize("overlap", [0, 1], ids=["in-stream", "overlapped"])
-def test_c4_twelve_packed_jobs_bursty_arrival(overlap):
-    from paper_2204_03211_b200 import binding as B
+def test_c4_twelve_packed_jobs_bursty_arrival_every_element(overlap):
     cfg = configs.c4()
-    pair = SampledPair(cfg, per_block=128, full_per_job=4)
+    pair = FullPair(cfg, overlap=overlap)       # the launch configuration bench.py times is "overlapped"
     try:
-        pair.svc.set_option(B.PS_OPT_OVERLAP, overlap)      # the launch configuration bench.py times is "overlapped"
-        stream = torch.cuda.Stream()
         for it in range(cfg.iterations):
             rounds = configs.rounds_for(cfg, it, 16)
-            assert all(len({j for j, _ in r}) >= 1 for r in rounds)
-            pair.iteration(it, rounds, stream)
-            pair.svc.join(stream)
-            stream.synchronize()
-        pair.compare(cfg.iterations)
+            pair.iteration(it, rounds)
+            if it in (0, cfg.iterations - 1):
+                assert pair.compare(it + 1) == cfg.num_params
         # one more iteration with everything ready at once: a single packed launch
         before = pair.svc.launch_info()["launches"]
-        pair.iteration(cfg.iterations, configs.rounds_all(cfg), stream)
-        pair.svc.join(stream)
-        stream.synchronize()
+        pair.iteration(cfg.iterations, configs.rounds_all(cfg))
         assert pair.svc.launch_info()["launches"] == before + 1
         pair.compare(cfg.iterations + 1)
     finally:
         pair.close()
 
 
-def test_c5_bert_large_shaped_adam_bf16_with_migration():
+def test_c5_bert_large_shaped_adam_bf16_with_migration_every_element():
     cfg = configs.c5()
-    pair = SampledPair(cfg, per_block=128, full_per_job=4)
+    pair = FullPair(cfg)
     try:
         rounds = configs.rounds_all(cfg)
         plan = configs.migration_plan(cfg)
         side = torch.cuda.Stream()
         for it in range(cfg.iterations):
             pair.iteration(it, rounds)
-            if it == 0:
-                pair.compare(1)
+            if it in (0, cfg.migrate_after, cfg.iterations - 1):     # first, first after the migration, last
+                assert pair.compare(it + 1) == cfg.num_params
             if it + 1 == cfg.migrate_after:
                 # a quarter of the blocks changes context between two iterations, on another stream
                 pair.migrate(plan, side)
-        pair.compare(cfg.iterations)
         used = [pair.svc.arena_info(c)[0] for c in range(cfg.num_contexts)]
         assert sum(used) == sum(3 * ((4 * b.nelem + 255) // 256 * 256) for b in cfg.jobs[0].blocks)
     finally:

@@ -342,5 +342,5 @@ def test_bench_replica_arm_two_ranks_on_one_device():
     cfg = configs.c1()
     assert line["n_gpus"] == 2 and line["scaling"] == "weak" and line["steps"] == 20
     assert abs(line["value"] - 2 * cfg.num_params / (line["ms_per_step"] * 1e-3)) <= 1e-6 * line["value"]
-    assert line["gpu_launches"] == 20 and line["cpu_baseline"] is None
+    assert line["gpu_launches"] == 20 * line["timed_region"]["blocks"] and line["cpu_baseline"] is None
     assert line["e2e"]["h2d_bytes_per_step"] == 4 * 4 * cfg.num_params
