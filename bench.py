@@ -475,11 +475,14 @@ def time_oracle(items, params, min_seconds: float, max_passes: int):
 # ------------------------------------------------------------------ block-sharded arm
 
 def sharded_main(args, cfg, config, rank, local_rank, world, device):
-    """One workload over `world` ranks: every block is owned by one rank, the
+    """One workload over `world` ranks: every block is owned by one rank; the
     W shards of a block are read in place from the worker ranks' exported
-    buffers (no collective in the path).  Total work is fixed: strong scaling."""
+    buffers, or copied into the owner's staging buffer ahead of the aggregate
+    (--transport); no collective in the path.  Total work is fixed: strong
+    scaling.  One JSON line per transport."""
     import torch.distributed as dist
-    from paper_2204_03211_b200 import sharded
+    import bench_sharded
+    from paper_2204_03211_b200 import binding as B
 
     def exchange(obj):
         got = [None] * world
@@ -487,48 +490,61 @@ def sharded_main(args, cfg, config, rank, local_rank, world, device):
         return got
 
     red_dev = device if args.dist_backend == "nccl" else None
-    wl = sharded.ShardedWorkload(cfg, rank, world, local_rank, exchange, dist.barrier, param_device=device)
-    from paper_2204_03211_b200 import binding as B
-    wl.sh.svc.set_option(B.PS_OPT_OVERLAP, int(not args.in_stream))
-    wl.fill(0, device)
-    n_sched = max(1, min(args.warmup, 8))      # every schedule runs once before the timed region
-    schedules = [configs.rounds_for(cfg, it, args.ticks) for it in range(n_sched)]
-    stream = torch.cuda.Stream(device)
+    transports = ["inplace", "staged"] if args.transport == "both" else [args.transport]
+    for transport in transports:
+        wl = bench_sharded.ShardedWorkload(cfg, rank, world, local_rank, exchange, dist.barrier, param_device=device,
+                                           transport=transport)
+        wl.sh.svc.set_option(B.PS_OPT_OVERLAP, int(not args.in_stream))
+        wl.fill(0, device)
+        n_sched = max(1, min(args.warmup, 8))
+        schedules = [configs.rounds_for(cfg, it, args.ticks) for it in range(n_sched)]
+        stream = torch.cuda.Stream(device)
 
-    def step(k, s):
-        n = wl.step(schedules[k % n_sched], s, key=k % n_sched)
-        if not args.in_stream:
-            wl.sh.svc.join(s)
-        return n
+        def step(k, s):
+            if transport == "staged":
+                wl.stage(s)
+                exchange(0)                  # host only: every rank's record call has been made
+                wl.wait_staged(s)
+            n = wl.step(schedules[k % n_sched], s, key=k % n_sched)
+            if not args.in_stream:
+                wl.sh.svc.join(s)
+            return n
 
-    for k in range(args.warmup):
-        step(k, stream)
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    ms, launches, host_ms = timed(lambda k, s: step(args.warmup + k, s), args.steps, stream, True, red_dev)
-    clocks = sampler.stop() if rank == 0 else {}
-    mine = [wl.owned_params, wl.owned_bytes, launches]
-    per_rank = exchange(mine)
-    if rank == 0:
-        value = cfg.num_params * args.steps / (ms * 1e-3)                     # every block once per step, all ranks
-        worst = max(r[1] for r in per_rank)
-        achieved = worst * args.steps / (ms * 1e-3) / 1e9                     # the most loaded rank's HBM traffic
-        peak, peak_kind = measured_peak()
-        config["parallelism"] = "blocks owned by %d ranks (longest-first partition), shards read in place from peers" % world
-        config["launch_mode"] = "in-stream" if args.in_stream else "overlapped, one ps_join per step"
-        print(json.dumps({
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "strong",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_source": peak_kind + " copy bandwidth",
-                         "note": "most loaded rank; with several GPUs the remote shards arrive over NVLink, "
-                                 "which bounds the step before HBM does"},
-            "per_rank": [{"params": r[0], "bytes_per_step": r[1], "launches": r[2]} for r in per_rank],
-            "cpu_baseline": None, "e2e": None, "gpu_launches": sum(r[2] for r in per_rank),
-            "host_ms_per_step": host_ms / args.steps, "clocks": clocks}))
-    wl.close()
+        sampler = ClockSampler(local_rank)
+        if rank == 0:
+            sampler.start()
+        for k in range(args.warmup):
+            step(k, stream)
+        torch.cuda.synchronize(device)
+        if rank == 0:
+            sampler.mark()
+        l0 = wl.sh.svc.launch_info()["launches"]
+        ms, rounds, host_ms = timed(lambda k, s: step(args.warmup + k, s), args.steps, stream, True, red_dev)
+        clocks = sampler.stop() if rank == 0 else {}
+        launches = wl.sh.svc.launch_info()["launches"] - l0
+        per_rank = exchange([wl.owned_params, wl.owned_bytes, launches, wl.nvlink_bytes_per_step])
+        if rank == 0:
+            value = cfg.num_params * args.steps / (ms * 1e-3)                     # every block once per step, all ranks
+            worst = max(r[1] for r in per_rank)
+            achieved = worst * args.steps / (ms * 1e-3) / 1e9                     # the most loaded rank's HBM traffic
+            peak, peak_kind = measured_peak()
+            cfg_out = dict(config)
+            cfg_out["parallelism"] = "blocks owned by %d ranks (longest-first partition); transport %s" % (
+                world, "in place: the owner's kernel reads the workers' buffers" if transport == "inplace" else
+                "staged: the workers copy their shards into the owner's memory ahead of the aggregate")
+            print(json.dumps({
+                "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "strong",
+                "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg_out, "transport": transport,
+                "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                             "traffic": None, "peak_source": peak_kind + " copy bandwidth",
+                             "note": "most loaded rank; with several GPUs the remote shards cross NVLink (read in "
+                                     "place by the kernel, or copied ahead of it), which bounds the step before HBM does"},
+                "per_rank": [{"params": r[0], "bytes_per_step": r[1], "launches": r[2],
+                              "nvlink_bytes_per_step": r[3]} for r in per_rank],
+                "cpu_baseline": None, "e2e": None, "gpu_launches": sum(r[2] for r in per_rank),
+                "host_ms_per_step": host_ms / args.steps, "clocks": clocks}))
+        wl.close()
     dist.destroy_process_group()
     return 0
 
@@ -615,6 +631,15 @@ def main():
     ap.add_argument("--shard-blocks", action="store_true",
                     help="with --gpus N > 1: ONE workload whose blocks are owned by the N ranks (strong scaling; "
                          "shards are read in place from the worker ranks' exported buffers) instead of N replicas")
+    ap.add_argument("--transport", default="both", choices=["inplace", "staged", "both"],
+                    help="with --shard-blocks: how a block's shards reach its owner (one JSON line per transport)")
+    ap.add_argument("--migration", action="store_true",
+                    help="instead of the aggregation benchmark: the overhead of migrating all blocks of a model "
+                         "between two contexts (bench_migration.py; its options follow)")
+    ap.add_argument("--models", default="alexnet,vgg16,awd_lm,bert_base")
+    ap.add_argument("--workers", type=int, default=2)
+    ap.add_argument("--reps", type=int, default=7)
+    ap.add_argument("--one-by-one", action="store_true", help="--migration: one ps_migrate_block call per block")
     ap.add_argument("--dist-backend", default="nccl", choices=["nccl", "gloo"],
                     help="process-group backend for the barriers and the max over ranks")
     ap.add_argument("--no-e2e", action="store_true")
@@ -623,6 +648,14 @@ def main():
                     help="skip timing the oracle on a bounded sample of each of the five configurations")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
+    if args.migration:
+        import bench_migration
+        if not torch.cuda.is_available():
+            raise SystemExit("needs a CUDA device")
+        torch.cuda.set_device(0)
+        for m in args.models.split(","):
+            print(json.dumps(bench_migration.one_model(m, args.workers, args.reps, args.one_by_one)))
+        return 0
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -1,6 +1,6 @@
 """Overhead of migrating ALL blocks of a job to another Aggregator context.
 
-    python -m paper_2204_03211_b200.migration_bench [--models alexnet,vgg16,awd_lm,bert_base] [--workers 2]
+    python bench.py --migration [--models alexnet,vgg16,awd_lm,bert_base] [--workers 2]
 
 The paper's counterpart is its table "Time overhead of migrating all tensors in
 a model" (Appendix B): what the training job sees when every tensor of a model
@@ -29,7 +29,7 @@ import sys
 import numpy as np
 import torch
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 

@@ -270,9 +270,10 @@ int ps_migrate_block(ps_service* svc, int job, int block, int dst_ctx, void* str
 
 /* The same for n blocks at once (host array of tasks, no block listed twice), as
  * ONE batch: every destination range is reserved first (PS_ERR_NOMEM leaves all
- * blocks where they were), one gather-copy kernel per 96 blocks moves the data
- * and one event marks the batch — moving all tensors of a model costs a few
- * launches instead of one copy call per tensor (the paper's Appendix B measures
+ * blocks where they were), one gather-copy kernel moves up to 1024 blocks (96
+ * where the driver refuses a 28 KB parameter block) and one event marks the
+ * batch — moving all tensors of a model costs one launch instead of one copy
+ * call per tensor (the paper's Appendix B measures
  * exactly that case: the overhead of migrating all tensors of a model).
  * Errors: BAD_ARG, DUPLICATE, NOMEM, NO_DEVICE, CUDA. */
 int ps_migrate_blocks(ps_service* svc, const ps_task* tasks, int n, int dst_ctx, void* stream);
@@ -473,6 +474,28 @@ int ps_peer_free(int device, void* dev_ptr);
 int ps_peer_open(int device, const unsigned char* handle, void** dev_ptr_out);
 int ps_peer_close(int device, void* dev_ptr);
 const char* ps_peer_last_error(void);
+
+/* Ordering between processes WITHOUT a host wait: interprocess events.  One
+ * process creates an event and passes its 64-byte handle on; the others open
+ * it.  ps_peer_event_record(event, stream) marks a point of the recorder's
+ * stream; ps_peer_event_wait(event, stream) makes a stream of any process wait
+ * for the most recent record — which must already have been ISSUED when the
+ * wait is enqueued (a wait on an event that nobody has recorded yet passes at
+ * once), so the waiter learns over a host channel that the record call has been
+ * made; it does not have to learn that the device has reached it.  Used for
+ * migration between services (the new owner's copy waits for the old owner's;
+ * paper Appendix B, "Data Consistency") and for staged pushes (the owner's
+ * aggregate waits for the workers' copies into its memory).  Events are
+ * destroyed by every process that holds them.
+ * ps_peer_copy_many enqueues n plain copies (copy engines) on `stream`;
+ * either side of each may be mapped peer memory.
+ * Errors: BAD_ARG, CUDA (text: ps_peer_last_error). */
+int ps_peer_event_create(int device, void** event_out, unsigned char* handle_out);
+int ps_peer_event_open(int device, const unsigned char* handle, void** event_out);
+int ps_peer_event_record(void* event, void* stream);
+int ps_peer_event_wait(void* event, void* stream);
+int ps_peer_event_destroy(void* event);
+int ps_peer_copy_many(int n, void* const* dsts, const void* const* srcs, const size_t* bytes, void* stream);
 
 /* Pull from another process (paper Section 4: Pull returns the current
  * parameters of (job, tensor)).  ps_arena_export writes the handle of a

@@ -125,6 +125,12 @@ _SIGNATURES = {
     "ps_peer_open": (C.c_int, [C.c_int, C.c_char_p, C.POINTER(C.c_void_p)]),
     "ps_peer_close": (C.c_int, [C.c_int, C.c_void_p]),
     "ps_peer_last_error": (C.c_char_p, []),
+    "ps_peer_event_create": (C.c_int, [C.c_int, C.POINTER(C.c_void_p), C.c_char_p]),
+    "ps_peer_event_open": (C.c_int, [C.c_int, C.c_char_p, C.POINTER(C.c_void_p)]),
+    "ps_peer_event_record": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "ps_peer_event_wait": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "ps_peer_event_destroy": (C.c_int, [C.c_void_p]),
+    "ps_peer_copy_many": (C.c_int, [C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ps_strerror": (C.c_char_p, [C.c_int]),
     "ps_last_cuda_error": (C.c_char_p, [C.c_void_p]),
     "ps_version": (C.c_char_p, []),
@@ -573,6 +579,37 @@ def ps_peer_open(device: int, handle: bytes) -> int:
 
 def ps_peer_close(device: int, ptr: int):
     _check_peer(load().ps_peer_close(device, ptr), "ps_peer_close")
+
+
+def ps_peer_event_create(device: int):
+    """Returns (event, 64-byte handle) of an event other processes can open."""
+    ev, handle = C.c_void_p(), C.create_string_buffer(PS_PEER_HANDLE_BYTES)
+    _check_peer(load().ps_peer_event_create(device, C.byref(ev), handle), "ps_peer_event_create")
+    return ev.value, handle.raw
+
+
+def ps_peer_event_open(device: int, handle: bytes) -> int:
+    ev = C.c_void_p()
+    _check_peer(load().ps_peer_event_open(device, handle, C.byref(ev)), "ps_peer_event_open")
+    return ev.value
+
+
+def ps_peer_event_record(event: int, stream=None):
+    _check_peer(load().ps_peer_event_record(event, _stream_ptr(stream)), "ps_peer_event_record")
+
+
+def ps_peer_event_wait(event: int, stream=None):
+    _check_peer(load().ps_peer_event_wait(event, _stream_ptr(stream)), "ps_peer_event_wait")
+
+
+def ps_peer_event_destroy(event: int):
+    _check_peer(load().ps_peer_event_destroy(event), "ps_peer_event_destroy")
+
+
+def ps_peer_copy_many(dsts, srcs, nbytes, stream=None):
+    """uint64 numpy arrays of destination and source addresses and of byte counts."""
+    _check_peer(load().ps_peer_copy_many(len(dsts), dsts.ctypes.data, srcs.ctypes.data, nbytes.ctypes.data,
+                                         _stream_ptr(stream)), "ps_peer_copy_many")
 
 
 def _bind(name):

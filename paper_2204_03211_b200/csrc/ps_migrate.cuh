@@ -1,29 +1,34 @@
-// Gather-copy kernel of block migration: moves up to kMigPerLaunch (source,
-// destination, bytes) ranges between context arenas in ONE launch (paper Section
-// 3.2 and Appendix B: the old Aggregator copies the tensor's contents — parameters
-// and metadata, here the optimizer state — to the new one).  Ranges are 256-byte
+// Gather-copy kernel of block migration: moves up to N (source, destination,
+// bytes) ranges between context arenas in ONE launch (paper Section 3.2 and
+// Appendix B: the old Aggregator copies the tensor's contents — parameters and
+// metadata, here the optimizer state — to the new one).  Ranges are 256-byte
 // aligned and a multiple of 256 bytes long (arena granularity); work is cut
-// into 64 KB tiles that CTAs take round-robin.
+// into 64 KB tiles that CTAs take round-robin.  The range table travels as a
+// kernel parameter: 96 ranges fit the 4 KB every driver accepts; the 1024-range
+// form (28 KB) uses the large parameter space of current drivers, so that all
+// blocks of a model move in one launch with no gap in the middle.
 #pragma once
 
 #include <cuda_runtime.h>
 
 namespace psb {
 
-constexpr int kMigPerLaunch = 96;
+constexpr int kMigSmall = 96, kMigLarge = 1024;
 constexpr unsigned int kMigTile = 65536;
 
-struct MigArgs {                       // passed by value (about 2.7 KB of kernel parameters)
-  const unsigned char* src[kMigPerLaunch];
-  unsigned char* dst[kMigPerLaunch];
-  unsigned long long bytes[kMigPerLaunch];
-  unsigned int tile_prefix[kMigPerLaunch + 1];   // first tile of each range; [n] = total tiles
+template <int N>
+struct MigArgs {                       // passed by value
+  const unsigned char* src[N];
+  unsigned char* dst[N];
+  unsigned long long bytes[N];
+  unsigned int tile_prefix[N + 1];     // first tile of each range; [n] = total tiles
   int n;
 };
 
 constexpr int kMigUnroll = 16;         // 128-bit loads in flight per thread: one 64 KB tile is one trip of 256 threads
 
-__global__ void __launch_bounds__(256) ps_migrate_kernel(const MigArgs a) {
+template <int N>
+__global__ void __launch_bounds__(256) ps_migrate_kernel(const __grid_constant__ MigArgs<N> a) {
   const unsigned int total = a.tile_prefix[a.n];
   for (unsigned int t = blockIdx.x; t < total; t += gridDim.x) {
     int lo = 0, hi = a.n;                          // largest d with tile_prefix[d] <= t

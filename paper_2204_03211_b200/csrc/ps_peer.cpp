@@ -74,6 +74,73 @@ int ps_peer_close(int device, void* dev_ptr) {
   return e == cudaSuccess ? PS_OK : fail(e);
 }
 
+// Interprocess events: how one process's stream waits for another process's copy
+// without either host waiting for its device.
+static_assert(sizeof(cudaIpcEventHandle_t) == PS_PEER_HANDLE_BYTES, "event handle size");
+
+int ps_peer_event_create(int device, void** event_out, unsigned char* handle_out) {
+  if (!event_out || !handle_out || device < 0) return PS_ERR_BAD_ARG;
+  *event_out = nullptr;
+  cudaError_t e = cudaSetDevice(device);
+  if (e != cudaSuccess) return fail(e);
+  cudaEvent_t ev = nullptr;
+  e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming | cudaEventInterprocess);
+  if (e != cudaSuccess) return fail(e);
+  cudaIpcEventHandle_t h;
+  e = cudaIpcGetEventHandle(&h, ev);
+  if (e != cudaSuccess) {
+    cudaEventDestroy(ev);
+    return fail(e);
+  }
+  std::memcpy(handle_out, &h, sizeof(h));
+  *event_out = ev;
+  return PS_OK;
+}
+
+int ps_peer_event_open(int device, const unsigned char* handle, void** event_out) {
+  if (!event_out || !handle || device < 0) return PS_ERR_BAD_ARG;
+  *event_out = nullptr;
+  cudaError_t e = cudaSetDevice(device);
+  if (e != cudaSuccess) return fail(e);
+  cudaIpcEventHandle_t h;
+  std::memcpy(&h, handle, sizeof(h));
+  cudaEvent_t ev = nullptr;
+  e = cudaIpcOpenEventHandle(&ev, h);
+  if (e != cudaSuccess) return fail(e);
+  *event_out = ev;
+  return PS_OK;
+}
+
+int ps_peer_event_record(void* event, void* stream) {
+  if (!event) return PS_ERR_BAD_ARG;
+  cudaError_t e = cudaEventRecord(static_cast<cudaEvent_t>(event), static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? PS_OK : fail(e);
+}
+
+int ps_peer_event_wait(void* event, void* stream) {
+  if (!event) return PS_ERR_BAD_ARG;
+  cudaError_t e = cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), static_cast<cudaEvent_t>(event), 0);
+  return e == cudaSuccess ? PS_OK : fail(e);
+}
+
+int ps_peer_event_destroy(void* event) {
+  if (!event) return PS_ERR_BAD_ARG;
+  cudaError_t e = cudaEventDestroy(static_cast<cudaEvent_t>(event));
+  return e == cudaSuccess ? PS_OK : fail(e);
+}
+
+int ps_peer_copy_many(int n, void* const* dsts, const void* const* srcs, const size_t* bytes, void* stream) {
+  if (n < 0 || (n > 0 && (!dsts || !srcs || !bytes))) return PS_ERR_BAD_ARG;
+  for (int i = 0; i < n; ++i) {
+    if (!bytes[i]) continue;
+    if (!dsts[i] || !srcs[i]) return PS_ERR_BAD_ARG;
+    // one plain copy per range, by the copy engines: the ranges may lie in a peer's memory
+    cudaError_t e = cudaMemcpyAsync(dsts[i], srcs[i], bytes[i], cudaMemcpyDefault, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail(e);
+  }
+  return PS_OK;
+}
+
 const char* ps_peer_last_error(void) { return g_peer_err.c_str(); }
 
 }  // extern "C"

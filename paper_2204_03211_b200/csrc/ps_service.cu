@@ -185,6 +185,7 @@ struct ps_service {
   std::vector<int> batch;                  // block indices, in arrival order
   unsigned long long batch_chunks = 0;     // their size in chunks of kChunkAuto elements
   long long opt_batch = 1;
+  bool mig_large_ok = true;                // the 28 KB kernel-parameter form of the migration kernel is accepted
   unsigned long long epoch = 0;            // bumped by whatever can invalidate a prepared round's table:
                                            // migration, import, unregistration, options
   int last_grid = 0, last_block = 0;
@@ -1501,22 +1502,45 @@ static int migrate_many(ps_service* s, const std::vector<int>& bis, int dst_ctx,
     e = cudaMemcpyAsync(s->ctxs[dst_ctx].base + moves[0].noff, s->ctxs[b.ctx].base + b.off, b.bytes,
                         cudaMemcpyDeviceToDevice, stream);
   } else {
-    for (size_t first = 0; first < moves.size() && e == cudaSuccess; first += kMigPerLaunch) {
-      MigArgs a;
-      a.n = (int)std::min<size_t>(kMigPerLaunch, moves.size() - first);
+    // one launch for up to 1024 blocks (a whole model); 96 at a time where the large
+    // kernel-parameter space is refused
+    auto launch_some = [&](auto* args, size_t first, size_t count) {
+      args->n = (int)count;
       unsigned int tiles = 0;
-      for (int k = 0; k < a.n; ++k) {
+      for (size_t k = 0; k < count; ++k) {
         Block& b = s->blocks[moves[first + k].bi];
-        a.src[k] = reinterpret_cast<const unsigned char*>(s->ctxs[b.ctx].base + b.off);
-        a.dst[k] = reinterpret_cast<unsigned char*>(s->ctxs[dst_ctx].base + moves[first + k].noff);
-        a.bytes[k] = b.bytes;
-        a.tile_prefix[k] = tiles;
+        args->src[k] = reinterpret_cast<const unsigned char*>(s->ctxs[b.ctx].base + b.off);
+        args->dst[k] = reinterpret_cast<unsigned char*>(s->ctxs[dst_ctx].base + moves[first + k].noff);
+        args->bytes[k] = b.bytes;
+        args->tile_prefix[k] = tiles;
         tiles += (unsigned int)((b.bytes + kMigTile - 1) / kMigTile);
       }
-      a.tile_prefix[a.n] = tiles;
-      const int grid = (int)std::min<unsigned int>(tiles, (unsigned int)s->num_sms * 16u);
-      ps_migrate_kernel<<<grid, 256, 0, stream>>>(a);
-      e = cudaGetLastError();
+      args->tile_prefix[count] = tiles;
+      return (int)std::min<unsigned int>(tiles, (unsigned int)s->num_sms * 16u);
+    };
+    size_t first = 0;
+    while (first < moves.size() && e == cudaSuccess) {
+      const size_t left = moves.size() - first;
+      if (left > (size_t)kMigSmall && s->mig_large_ok) {
+        static thread_local MigArgs<kMigLarge> big;
+        const size_t count = std::min<size_t>(kMigLarge, left);
+        const int grid = launch_some(&big, first, count);
+        ps_migrate_kernel<kMigLarge><<<grid, 256, 0, stream>>>(big);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) {            // refused at launch: nothing ran; remember and take the small form
+          s->mig_large_ok = false;
+          e = cudaSuccess;
+          continue;
+        }
+        first += count;
+      } else {
+        MigArgs<kMigSmall> small;
+        const size_t count = std::min<size_t>(kMigSmall, left);
+        const int grid = launch_some(&small, first, count);
+        ps_migrate_kernel<kMigSmall><<<grid, 256, 0, stream>>>(small);
+        e = cudaGetLastError();
+        first += count;
+      }
     }
   }
   if (e == cudaSuccess) e = cudaEventRecord(s->batches[batch].ev, stream);

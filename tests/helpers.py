@@ -95,6 +95,21 @@ class Pair:
         v = self.svc.view(s1, n).cpu().numpy() if s1 else None
         return p, a, v, ctx
 
+    def check_padding(self, j: int, b: int, nelem: int, sections: int, tag: str):
+        """Every section of a block's arena range (parameters, state) is rounded
+        up to 256 bytes and zeroed at registration; the kernels may never write
+        past the last element, so the bytes between 4*nelem and the end of each
+        section are still zero (a short overrun would not show in any other
+        comparison)."""
+        _, _, sec = self.svc.block_location(j, b)
+        pad = (sec - 4 * nelem) // 4
+        if pad == 0:
+            return
+        base = self.svc.pull(j, b)
+        for k in range(sections):
+            tail = self.svc.view(base + k * sec + 4 * nelem, pad).view(torch.int32)
+            assert int(tail.abs().max()) == 0, "%s: bytes after section %d were written" % (tag, k)
+
     def compare(self, sq_rtol: float = 1e-5, exact: bool = True):
         worst = 0.0
         assert self.svc.device_status() == 0, "a bounded wait expired inside a kernel"
@@ -118,6 +133,7 @@ class Pair:
                 assert step == rstep, tag + " step"
                 assert abs(sq - rsq) <= sq_rtol * abs(rsq) + 1e-300, tag + " sqnorm %r vs %r" % (sq, rsq)
                 worst = max(worst, float(np.max(np.abs(p.astype(np.float64) - rp))))
+                self.check_padding(j, b.block, b.nelem, 3 if rv is not None else 2, tag)
         return worst
 
 

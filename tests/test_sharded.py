@@ -5,10 +5,12 @@ CPU: the ownership map (balanced, deterministic, identical on every rank) and
 the per-rank registry, with two gloo ranks over planning-only services.
 GPU: two processes sharing one device, each the owner of half the blocks and
 the host of half the workers; shards are read in place from the other
-process's exported buffer (CUDA IPC), blocks change owner between two
-iterations (export, import, unregister) and every owned block is compared bit
-for bit with the CPU oracle.  The two ranks' kernels never wait on one another:
-the ranks meet only in host barriers."""
+process's exported buffer (CUDA IPC) or copied into the owner's staging buffer
+ahead of the aggregate; blocks change owner between two aggregates with no host
+waiting for its device in between (export, import and the next aggregate are
+ordered by interprocess events and the library's own); every owned block is
+compared bit for bit with the CPU oracle.  The two ranks' kernels never wait on
+one another: ranks meet in host exchanges, streams wait on events."""
 import json
 import os
 import socket
@@ -24,6 +26,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 sys.path.insert(0, ROOT)
 sys.path.insert(0, os.path.join(ROOT, "tests"))
 
+import bench_sharded  # noqa: E402
 from paper_2204_03211_b200 import binding as B, sharded  # noqa: E402
 from workload import configs  # noqa: E402
 
@@ -115,7 +118,7 @@ def test_two_gloo_ranks_agree_on_owners_and_split_the_registry(tmp_path):
         assert abs(got["elems"][0] - got["elems"][1]) <= 0.02 * cfg.num_params
 
 
-def _gpu_rank(rank, world, port, out):
+def _gpu_rank(rank, world, port, out, transport="inplace"):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
     dist.init_process_group("gloo", rank=rank, world_size=world)
     from helpers import oracle_hp, tiny_config, to_np
@@ -131,7 +134,8 @@ def _gpu_rank(rank, world, port, out):
     a = tiny_config([70001, 5, 4096, 300000, 33], 3).jobs[0]
     b = tiny_config([1 << 18, 12289, 1, 8192], 4, opt=configs.ADAM, grad_dtype=configs.BF16).jobs[0]
     cfg = configs.Config("sharded-tiny", 321, 3, [a, b])
-    wl = sharded.ShardedWorkload(cfg, rank, world, 0, exchange, dist.barrier, arena_slack=16 << 20)   # room for adopted blocks
+    wl = bench_sharded.ShardedWorkload(cfg, rank, world, 0, exchange, dist.barrier, arena_slack=16 << 20,   # room for adopted blocks
+                                       transport=transport)
     # the oracle of each rank follows EVERY block (they are tiny), so that a block
     # adopted by this rank half-way has its history
     ora = A.OracleAggregator(1, 0)
@@ -143,20 +147,10 @@ def _gpu_rank(rank, world, port, out):
     every = configs.rounds_all(cfg)[0]
     rounds = [every[:4], every[4:]]
     remote_reads, adopted, sent = 0, set(), 0
-    for it in range(3):
-        if it == 2:
-            # between two iterations every rank hands its two lowest blocks of each job to the other rank
-            owner0 = dict(wl.sh.owner)
-            moves = []
-            for r in range(world):
-                for j in range(len(cfg.jobs)):
-                    theirs = sorted(blk for (jj, blk), o in owner0.items() if jj == j and o == r)
-                    moves += [(j, blk, 1 - r) for blk in theirs[:2]]
-            before = set(wl.sh.owned(every))
-            sent = wl.migrate(moves, exchange)
-            adopted = set(wl.sh.owned(every)) - before
-        wl.fill(it, "cpu")
-        assert wl.step(rounds, key=0) >= 1
+    stream = torch.cuda.Stream()
+
+    def oracle_iteration(it):
+        nonlocal remote_reads
         for j, job in enumerate(cfg.jobs):
             host = to_np(generate.grad_slab(cfg, j, it))
             for blk in job.blocks:
@@ -165,8 +159,41 @@ def _gpu_rank(rank, world, port, out):
                     if wl.sh.owns(j, blk.block):
                         remote_reads += int(sharded.worker_rank(w, world) != rank)
         ora.aggregate(every)
+
+    def device_iteration():
+        if transport == "staged":
+            wl.stage(stream)
+            exchange(0)                                            # every rank's record call has been made
+            wl.wait_staged(stream)
+        assert wl.step(rounds, stream, key=0) >= 1
+
+    for it in range(3):
+        wl.fill(it, "cpu")
+        device_iteration()
+        oracle_iteration(it)
+        if it == 1 and transport == "inplace":
+            # Every rank hands its two lowest blocks of each job to the other rank RIGHT AFTER enqueueing
+            # iteration 1's aggregates, and the next aggregates (the same gradient buffers once more, so that
+            # nothing has to be refilled and nobody synchronizes) follow at once: the copies wait for the
+            # aggregates, the imports for the exports, the new owner's aggregates for the imports — all on
+            # the devices' side.
+            owner0 = dict(wl.sh.owner)
+            moves = []
+            for r in range(world):
+                for j in range(len(cfg.jobs)):
+                    theirs = sorted(blk for (jj, blk), o in owner0.items() if jj == j and o == r)
+                    moves += [(j, blk, 1 - r) for blk in theirs[:2]]
+            before = set(wl.sh.owned(every))
+            sent = wl.migrate(moves, exchange, stream)
+            adopted = set(wl.sh.owned(every)) - before
+            device_iteration()
+            oracle_iteration(it)
+            sent += wl.migrate([(j, blk, 1 - r) for (j, blk, r) in moves[:2]], exchange, stream)   # and two of them back
+            device_iteration()
+            oracle_iteration(it)
         torch.cuda.synchronize()
         dist.barrier()                                             # every rank has read the buffers: refill allowed
+    steps_done = 5 if transport == "inplace" else 3
     ok, checked = True, 0
     for (j, blk) in wl.sh.owned(every):
         n = cfg.jobs[j].blocks[blk].nelem
@@ -179,7 +206,7 @@ def _gpu_rank(rank, world, port, out):
             ok &= np.array_equal(wl.sh.svc.view(s1, n).cpu().numpy(), rv)
         sq, step = wl.sh.svc.block_stats(j, blk)
         rsq, rstep = ora.block_stats(j, blk)
-        ok &= step == rstep == 3 and abs(sq - rsq) <= 1e-5 * abs(rsq) + 1e-300
+        ok &= step == rstep == steps_done and abs(sq - rsq) <= 1e-5 * abs(rsq) + 1e-300
         checked += 1
     # Pull across ranks: the other rank's blocks, read in place from its mapped arena
     wl.open_arenas(exchange)
@@ -201,7 +228,7 @@ def _gpu_rank(rank, world, port, out):
             ok &= e.status == B.PS_ERR_BAD_ARG
     with open(out % rank, "w") as f:
         json.dump({"ok": bool(ok), "checked": checked, "pulled": pulled, "remote_reads": remote_reads, "adopted": len(adopted),
-                   "sent": sent, "status": wl.sh.svc.device_status()}, f)
+                   "sent": sent, "status": wl.sh.svc.device_status(), "nvlink": wl.nvlink_bytes_per_step}, f)
     wl.close()
     dist.barrier()
     dist.destroy_process_group()
@@ -217,6 +244,20 @@ def test_two_processes_on_one_device_read_each_others_shards_in_place(tmp_path):
     assert all(g["checked"] + g["pulled"] == 9 for g in got)       # the rest was pulled from the other rank's arena
     assert all(g["remote_reads"] > 0 for g in got)                 # each rank consumed shards hosted by the other
     assert all(g["adopted"] >= 2 and g["sent"] > 0 for g in got)   # and blocks changed owner in both directions
+
+
+@pytest.mark.gpu
+def test_two_processes_on_one_device_staged_transport(tmp_path):
+    """The same deployment with the workers' shards COPIED into the owner's
+    staging buffer ahead of every aggregate (interprocess events order the
+    owner's launch after the copies): same results, and the owners' kernels read
+    nothing but their own memory."""
+    out = str(tmp_path / "s%d.json")
+    mp.spawn(_gpu_rank, args=(2, _free_port(), out, "staged"), nprocs=2, join=True)
+    got = [json.load(open(out % r)) for r in range(2)]
+    assert all(g["ok"] and g["status"] == 0 for g in got), got
+    assert sum(g["checked"] for g in got) == 9 and all(g["checked"] + g["pulled"] == 9 for g in got)
+    assert all(g["nvlink"] > 0 for g in got)                       # each rank sent shards to the other
 
 
 @pytest.mark.gpu

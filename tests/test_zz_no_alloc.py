@@ -7,7 +7,8 @@ allocation may bring — so its scratch lives in a fixed array inside the
 library.  Here the same block is aggregated twice in a row (steps 1 and 2)
 through a ps_service and through the no-allocation call, on identical inputs;
 parameters and optimizer state must agree bit for bit (both run the same
-kernel) and the gradient norm within the tolerance the other tests use.
+kernel) and the gradient norm within the tolerance the other tests use.  The
+CPU oracle is the second, independent checker of the same two calls.
 
 The file name sorts last on purpose: a run that stops at the first failure has
 already been through every other test.  It also passes on its own in a fresh
@@ -17,6 +18,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import aggregator as A
 from paper_2204_03211_b200 import binding as B
 
 pytestmark = pytest.mark.gpu
@@ -51,9 +53,17 @@ def test_no_alloc_entry_matches_service_two_calls_in_a_row(opt, dtype, W, nelem)
         sq = torch.full((1,), -1.0, device="cuda", dtype=torch.float64)
         stream = torch.cuda.Stream()
         torch.cuda.synchronize()
+        # the oracle's copy of the same block
+        hp = A.HParams(opt, dtype, W, d.lr, d.momentum, d.weight_decay, d.beta1, d.beta2, d.eps, d.grad_scale)
+        op = p0.cpu().numpy().copy()
+        o0 = np.zeros(nelem, np.float32)
+        o1 = np.zeros(nelem, np.float32) if opt == B.PS_ADAM else None
         for step in (1, 2):
             shards = [(torch.randn(nelem, device="cuda", generator=gen) * 1e-2).to(gdt) for _ in range(W)]
             torch.cuda.synchronize()
+            host = [g.view(torch.int16).cpu().numpy().view(np.uint16) if dtype == B.PS_BF16 else g.cpu().numpy()
+                    for g in shards]
+            osq = A.block_step(hp, step, host, op, o0, o1)
             for w, g in enumerate(shards):
                 svc.push(j, 0, w, g)
             svc.aggregate([(j, 0)], stream)
@@ -68,8 +78,44 @@ def test_no_alloc_entry_matches_service_two_calls_in_a_row(opt, dtype, W, nelem)
             ref_sq, ref_step = svc.block_stats(j, 0)
             assert ref_step == step
             assert abs(sq.item() - ref_sq) <= 1e-5 * abs(ref_sq)
+            # and against the oracle
+            assert np.array_equal(p.cpu().numpy(), op), "parameters differ from the oracle at step %d" % step
+            assert np.array_equal(s0.cpu().numpy(), o0)
+            if s1 is not None:
+                assert np.array_equal(s1.cpu().numpy(), o1)
+            assert abs(sq.item() - osq) <= 1e-5 * abs(osq)
     finally:
         svc.close()
+
+
+def test_norm_output_needs_only_eight_byte_alignment():
+    """The norm is one double written by one thread: an output that is 8- but
+    not 16-byte aligned (element 1 of a double tensor) is accepted and does not
+    change the result (nor push the block onto the scalar path)."""
+    torch.cuda.set_device(0)
+    nelem, W = 200_000, 4
+    gen = torch.Generator(device="cuda").manual_seed(99)
+    d = _desc(B.PS_SGD, B.PS_F32, W)
+    p0 = torch.randn(nelem, device="cuda", generator=gen) * 0.05
+    shards = [torch.randn(nelem, device="cuda", generator=gen) * 1e-2 for _ in range(W)]
+    out = torch.full((4,), -1.0, device="cuda", dtype=torch.float64)
+    assert out.data_ptr() % 16 == 0
+    results = []
+    for k in (0, 1):                       # 16-byte aligned, then 8-byte aligned only
+        p, s0 = p0.clone(), torch.zeros(nelem, device="cuda")
+        torch.cuda.synchronize()
+        B.ps_aggregate_block_noalloc(d, 1, nelem, p, s0, None, shards, out.data_ptr() + 8 * k)
+        torch.cuda.synchronize()
+        results.append((p.cpu().numpy(), s0.cpu().numpy(), float(out[k])))
+    assert np.array_equal(results[0][0], results[1][0]) and np.array_equal(results[0][1], results[1][1])
+    assert results[0][2] == results[1][2] > 0
+    hp = A.HParams(B.PS_SGD, B.PS_F32, W, d.lr, d.momentum, d.weight_decay, d.beta1, d.beta2, d.eps, d.grad_scale)
+    op, o0 = p0.cpu().numpy().copy(), np.zeros(nelem, np.float32)
+    osq = A.block_step(hp, 1, [g.cpu().numpy() for g in shards], op, o0)
+    assert np.array_equal(results[1][0], op) and np.array_equal(results[1][1], o0)
+    assert abs(results[1][2] - osq) <= 1e-5 * osq
+    with pytest.raises(ValueError):
+        B.ps_aggregate_block_noalloc(d, 1, nelem, p0.clone(), torch.zeros(nelem, device="cuda"), None, shards[:3])
 
 
 def test_no_alloc_entry_rejects_what_it_cannot_hold():
