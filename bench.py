@@ -266,98 +266,109 @@ class Workload:
     # ---- end to end: host gradients in, host parameters out
 
     def prepare_host(self, pool_bytes: int):
-        total = sum(s.numel() * s.element_size() for s in self.slabs)
-        pool_bytes = min(pool_bytes, total)
-        self.pool = torch.empty(pool_bytes // 4, dtype=torch.float32).pin_memory()
-        # fill the pool with the same gradient bits (device -> host copy of the slabs' head)
-        flat = self.pool.view(torch.uint8)
+        """Pinned host memory holding every worker's shard of every block in the
+        layout ps_push_host_batch sends as few copies: job after job, block
+        after block in id order, worker after worker, rows padded to 256 bytes.
+        If the pool is smaller than the workload's gradients, later jobs reuse
+        the pool from its start (the bytes that cross the link are the same)."""
+        cfg = self.cfg
+        job_bytes, row = [], {}
+        for j, job in enumerate(cfg.jobs):
+            esz = 2 if job.grad_dtype == configs.BF16 else 4
+            tot = 0
+            for b in job.blocks:
+                row[(j, b.block)] = (b.nelem * esz + 255) // 256 * 256
+                tot += row[(j, b.block)] * job.num_workers
+            job_bytes.append(tot)
+        total = sum(job_bytes)
+        pool_bytes = max(min(pool_bytes, total), max(job_bytes))
+        self.pool = torch.empty(pool_bytes, dtype=torch.uint8, pin_memory=True)
+        # gradient bit patterns (device -> host copy of the slabs' first bytes, repeated)
         off = 0
-        for s in self.slabs:
-            src = (s._base if s._base is not None else s).view(-1).view(torch.uint8)
-            n = min(src.numel(), flat.numel() - off)
+        for sl in self.slabs:
+            src = (sl._base if sl._base is not None else sl).view(-1).view(torch.uint8)
+            n = min(src.numel(), pool_bytes - off)
             if n <= 0:
                 break
-            flat[off:off + n].copy_(src[:n])
+            self.pool[off:off + n].copy_(src[:n])
             off += n
-        self.out = torch.empty(self.cfg.num_params, dtype=torch.float32).pin_memory()
+        while 0 < off < pool_bytes:
+            n = min(off, pool_bytes - off)
+            self.pool[off:off + n].copy_(self.pool[:n])
+            off += n
+        base, start, self.host_ptr = self.pool.data_ptr(), 0, {}
+        for j, job in enumerate(cfg.jobs):
+            if start + job_bytes[j] > pool_bytes:
+                start = 0
+            cur = start
+            for b in job.blocks:
+                for w in range(job.num_workers):
+                    self.host_ptr[(j, b.block, w)] = base + cur
+                    cur += row[(j, b.block)]
+            start = cur
+        self.out = torch.empty(cfg.num_params, dtype=torch.float32, pin_memory=True)
         self.pool_bytes = pool_bytes
         self.pull_stream = torch.cuda.Stream(torch.device("cuda", self.device))
         self.pull_done = torch.cuda.Event()
-        self.h2d = total
-        self.d2h = self.cfg.num_params * 4
+        self.h2d = sum(job.num_params * job.num_workers * (2 if job.grad_dtype == configs.BF16 else 4)
+                       for job in cfg.jobs)
+        self.d2h = cfg.num_params * 4
         self._out_off, acc = {}, 0
-        for j, job in enumerate(self.cfg.jobs):
+        for j, job in enumerate(cfg.jobs):
             self._out_off[j] = acc
             acc += job.num_params
+        # call arguments per schedule and round: the host addresses of the round's shards
+        self.host_args = []
+        for rounds in self.schedules:
+            per_round = []
+            for r in rounds:
+                ptrs = np.array([self.host_ptr[(int(j), int(b), int(w))]
+                                 for j, b, w in zip(r["jobs"], r["blocks"], r["workers"])], np.uint64)
+                outs = [(j, b, self.out.data_ptr() + 4 * (self._out_off[j] + cfg.jobs[j].blocks[b].job_offset))
+                        for (j, b) in r["ready"]]
+                per_round.append((ptrs, outs))
+            self.host_args.append(per_round)
 
-    def step_host(self, k: int, stream) -> int:
-        svc, cfg = self.svc, self.cfg
-        rounds = self.schedules[k % len(self.schedules)]
-        pool_ptr, pool_bytes = self.pool.data_ptr(), self.pool_bytes
-        cursor = 0
-        out_ptr = self.out.data_ptr()
-        out_off = {}
-        acc = 0
-        for j, job in enumerate(cfg.jobs):
-            out_off[j] = acc
-            acc += job.num_params
-        for r in rounds:
-            for (j, b) in r["ready"]:
-                job = cfg.jobs[j]
-                nbytes = job.blocks[b].nelem * (2 if job.grad_dtype == configs.BF16 else 4)
-                for w in range(job.num_workers):
-                    if cursor + nbytes > pool_bytes:
-                        cursor = 0
-                    svc.push_host(j, b, w, pool_ptr + cursor, stream)
-                    cursor += (nbytes + 255) // 256 * 256
-            svc.aggregate(r["tasks"], stream)
-            # parameters travel back on a second stream (the library orders each copy after the
-            # block's aggregate), so device-to-host traffic overlaps the next round's uploads
-            for (j, b) in r["ready"]:
-                svc.pull_host(j, b, out_ptr + 4 * (out_off[j] + cfg.jobs[j].blocks[b].job_offset), self.pull_stream)
+    def _pull_round(self, outs):
+        # parameters travel back on a second stream (the library orders each copy after the
+        # block's aggregate), so device-to-host traffic overlaps the next round's uploads
+        svc, ps = self.svc, self.pull_stream
+        for (j, b, dst) in outs:
+            svc.pull_host(j, b, dst, ps)
+
+    def _end_host_step(self, stream):
         self.pull_done.record(self.pull_stream)
         stream.wait_event(self.pull_done)           # the step ends when its last result is on the host
         if self.overlap:
-            svc.join(stream)
-        return len(rounds)
+            self.svc.join(stream)
 
+    def step_host(self, k: int, stream) -> int:
+        """End to end, staged: the round's shards are copied from pinned host
+        memory into device staging (ps_push_host_batch: neighbours travel as one
+        copy), aggregated, and the parameters copied back to the host."""
+        svc = self.svc
+        sched = k % len(self.schedules)
+        rounds = self.schedules[sched]
+        for r, (ptrs, outs) in zip(rounds, self.host_args[sched]):
+            svc.push_host_batch(r["jobs"], r["blocks"], r["workers"], ptrs, stream)
+            svc.aggregate(r["tasks"], stream)
+            self._pull_round(outs)
+        self._end_host_step(stream)
+        return len(rounds)
 
     def step_host_mapped(self, k: int, stream) -> int:
         """End to end without staging copies: pinned host memory is addressable
         from the device, so the pinned shards are pushed as they are and the
         aggregation kernel reads them over PCIe in place; parameters return to
         the host as in step_host."""
-        svc, cfg = self.svc, self.cfg
-        rounds = self.schedules[k % len(self.schedules)]
-        if not hasattr(self, "_mapped_args"):
-            self._mapped_args = {}
-        out_ptr = self.out.data_ptr()
-        for i, r in enumerate(rounds):
-            key = (k % len(self.schedules), i)
-            if key not in self._mapped_args:
-                # where each (block, worker) shard of this round sits in the pinned pool
-                jobs, blocks, workers, ptrs = [], [], [], []
-                cursor = 0
-                for (j, b) in r["ready"]:
-                    job = cfg.jobs[j]
-                    nbytes = job.blocks[b].nelem * (2 if job.grad_dtype == configs.BF16 else 4)
-                    for w in range(job.num_workers):
-                        if cursor + nbytes > self.pool_bytes:
-                            cursor = 0
-                        jobs.append(j); blocks.append(b); workers.append(w)
-                        ptrs.append(self.pool.data_ptr() + cursor)
-                        cursor += (nbytes + 255) // 256 * 256
-                self._mapped_args[key] = (np.array(jobs, np.int32), np.array(blocks, np.int32),
-                                          np.array(workers, np.int32), np.array(ptrs, np.uint64))
-            svc.push_batch(*self._mapped_args[key])
+        svc = self.svc
+        sched = k % len(self.schedules)
+        rounds = self.schedules[sched]
+        for r, (ptrs, outs) in zip(rounds, self.host_args[sched]):
+            svc.push_batch(r["jobs"], r["blocks"], r["workers"], ptrs)
             svc.aggregate(r["tasks"], stream)
-            for (j, b) in r["ready"]:
-                svc.pull_host(j, b, out_ptr + 4 * (self._out_off[j] + cfg.jobs[j].blocks[b].job_offset),
-                              self.pull_stream)
-        self.pull_done.record(self.pull_stream)
-        stream.wait_event(self.pull_done)
-        if self.overlap:
-            svc.join(stream)
+            self._pull_round(outs)
+        self._end_host_step(stream)
         return len(rounds)
 
 
@@ -611,7 +622,8 @@ def main():
                     help="staged: only the e2e leg whose shards are copied into device staging; mapped: "
                          "also a second leg (e2e_mapped) whose pinned shards are pushed as they are and read by "
                          "the kernel over PCIe")
-    ap.add_argument("--host-pool-gb", type=float, default=8.0)
+    ap.add_argument("--host-pool-gb", type=float, default=24.0,
+                    help="upper bound on the pinned host memory of the end-to-end legs (at least the largest job's shards)")
     ap.add_argument("--jobs", default="", help="comma-separated subset of the workload's jobs (profiling a small case)")
     ap.add_argument("--first-blocks", type=int, default=0, help="keep only the first N blocks of every job")
     ap.add_argument("--chunk-elems", type=int, default=0, help="PS_OPT_CHUNK_ELEMS (0 = automatic)")

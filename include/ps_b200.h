@@ -202,6 +202,21 @@ int ps_push_batch(ps_service* svc, int n, const int* jobs, const int* blocks, co
 int ps_push_host(ps_service* svc, int job, int block, int worker, const void* grad_host_ptr,
                  void* stream);
 
+/* n pushes from host memory in one call (host arrays of length n), all-or-nothing.
+ * The staging buffers of a job's blocks are ONE device region, laid out block after
+ * block in id order, each block W rows of round_up(nelem * element size, 256) bytes
+ * (allocated at the job's first push from host memory, for the blocks it has then).
+ * Shards that lie in the caller's host buffer in that same layout — block after
+ * block, worker after worker, rows padded to 256 bytes — are neighbours on both
+ * sides and are sent as ONE copy, padding included: a round of many small tensors
+ * then costs a few large copies instead of one small copy per (block, worker).
+ * Any other host layout works too, with one copy per shard.  The host buffers must
+ * stay valid until the copies complete; the ps_aggregate that consumes the pushes
+ * is enqueued on the same stream (or one ordered after it).
+ * Errors: those of ps_push_host; DUPLICATE also for a (block, worker) listed twice. */
+int ps_push_host_batch(ps_service* svc, int n, const int* jobs, const int* blocks, const int* workers,
+                       const void* const* grad_host_ptrs, void* stream);
+
 /* Aggregates every task in `ready` (host array, any mix of jobs) in ONE kernel
  * launch on `stream`: sum of the W shards in worker order, optimizer update of
  * the master copy and state, per-block squared gradient norm (the paper's

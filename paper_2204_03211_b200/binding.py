@@ -67,6 +67,7 @@ _SIGNATURES = {
     "ps_push_rows_batch": (C.c_int, [C.c_void_p, C.c_int] + [C.c_void_p] * 7),
     "ps_push_batch": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ps_push_host": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
+    "ps_push_host_batch": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ps_aggregate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "ps_join": (C.c_int, [C.c_void_p, C.c_void_p]),
     "ps_flush": (C.c_int, [C.c_void_p]),
@@ -238,6 +239,12 @@ def ps_push_batch(svc, jobs, blocks, workers, ptrs):
 
 def ps_push_host(svc, job: int, block: int, worker: int, grad_host, stream=None):
     _check(load().ps_push_host(svc, job, block, worker, _ptr(grad_host), _stream_ptr(stream)), "ps_push_host", svc)
+
+
+def ps_push_host_batch(svc, jobs, blocks, workers, host_ptrs, stream=None):
+    """jobs/blocks/workers: int32 numpy arrays; host_ptrs: uint64 numpy array of host addresses."""
+    _check(load().ps_push_host_batch(svc, len(jobs), jobs.ctypes.data, blocks.ctypes.data, workers.ctypes.data,
+                                     host_ptrs.ctypes.data, _stream_ptr(stream)), "ps_push_host_batch", svc)
 
 
 def make_tasks(pairs):
@@ -623,7 +630,7 @@ def _bind(name):
     return method
 
 
-for _n in ("flush", "round", "round_prepare", "round_run", "round_release", "launch_stats", "registry_info", "register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "aggregate", "join", "pull", "pull_batch", "pull_host",
+for _n in ("flush", "round", "round_prepare", "round_run", "round_release", "launch_stats", "registry_info", "register_job", "register_block", "push", "push_rows", "push_rows_batch", "push_batch", "push_host", "push_host_batch", "aggregate", "join", "pull", "pull_batch", "pull_host",
            "migrate_block", "migrate_blocks", "block_stats", "block_profile", "job_profile", "block_state", "plan", "set_option", "get_option", "arena_info",
            "launch_info", "device_status", "block_export", "block_import", "unregister_block", "arena_export", "block_location"):
     setattr(Service, _n, _bind(_n))

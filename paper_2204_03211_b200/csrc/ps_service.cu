@@ -39,6 +39,8 @@ struct Job {
   std::vector<int> block_of_id;            // block id -> index into Service::blocks, -1 = none
   mutable unsigned long long bc_step = 0;  // step the cached Adam scalars belong to
   mutable float bc_ss = 0.f, bc_sbc2 = 0.f;
+  char* stage_base = nullptr;              // staging region of the job's blocks for pushes from host memory
+  size_t stage_bytes = 0;
   size_t grad_esize() const { return d.grad_dtype == PS_BF16 ? 2 : 4; }
   int nstate() const { return d.opt == PS_ADAM ? 2 : 1; }
 };
@@ -63,8 +65,9 @@ struct Block {
   int last_slot = -1;                      // slot of the last aggregate
   unsigned long long last_slot_gen = 0;
   int mig_batch = -1;                      // migration batch whose copy may still be in flight
-  void* staging = nullptr;                 // device buffer for ps_push_host
+  void* staging = nullptr;                 // device buffer for ps_push_host: W rows of staging_row bytes
   size_t staging_row = 0;
+  bool staging_own = false;                // its own allocation (else a range of the job's staging region)
 };
 
 struct Ctx {
@@ -720,7 +723,9 @@ int ps_destroy(ps_service* s) {
     flush_batch(s);
     cudaDeviceSynchronize();
     for (auto& b : s->blocks)
-      if (b.staging) cudaFree(b.staging);
+      if (b.staging && b.staging_own) cudaFree(b.staging);
+    for (auto& j : s->jobs)
+      if (j.stage_base) cudaFree(j.stage_base);
     for (auto& m : s->batches)
       if (m.ev) cudaEventDestroy(m.ev);
     for (auto& sl : s->slots) {
@@ -931,36 +936,126 @@ int ps_push_batch(ps_service* s, int n, const int* jobs, const int* blocks, cons
   return push_batch_locked(s, n, jobs, blocks, workers, ptrs);
 }
 
-int ps_push_host(ps_service* s, int job, int block, int worker, const void* host_ptr, void* stream) {
-  if (!alive(s)) return PS_ERR_BAD_HANDLE;
-  std::lock_guard<std::mutex> lk(s->mu);
-  Block* b = nullptr;
-  int rc = push_checked(s, job, block, worker, host_ptr, &b, false);
-  if (rc) return rc;
-  if (!has_device(s)) return PS_ERR_NO_DEVICE;
-  PS_CUDA(s, cudaSetDevice(s->device));
-  const Job& j = s->jobs[b->job];
-  if (!b->staging) {
-    b->staging_row = Arena::round_up(b->nelem * j.grad_esize());
-    cudaError_t e = cudaMalloc(&b->staging, b->staging_row * j.d.num_workers);
+// Gives block b a staging buffer for pushes from host memory.  The first such push
+// of a job allocates ONE region for all blocks the job has then, laid out block after
+// block in id order, each block W rows of round_up(nelem * element size, 256) bytes:
+// shards that are neighbours in the caller's host buffer in that same layout are then
+// neighbours on the device too and travel as one copy.  Blocks registered later get
+// an allocation of their own.
+static int ensure_staging(ps_service* s, Block& b) {
+  if (b.staging) return PS_OK;
+  Job& j = s->jobs[b.job];
+  const size_t W = (size_t)j.d.num_workers;
+  if (!j.stage_base) {
+    size_t total = 0;
+    for (int bi : j.block_of_id)
+      if (bi >= 0) total += Arena::round_up(s->blocks[bi].nelem * j.grad_esize()) * W;
+    void* base = nullptr;
+    cudaError_t e = cudaMalloc(&base, total ? total : 256);
     if (e != cudaSuccess) {
-      b->staging = nullptr;
       cudaGetLastError();
       if (e == cudaErrorMemoryAllocation) return PS_ERR_NOMEM;
       s->cuda_err = cudaGetErrorString(e);
       return PS_ERR_CUDA;
     }
+    j.stage_base = static_cast<char*>(base);
+    j.stage_bytes = total;
+    size_t off = 0;
+    for (int bi : j.block_of_id) {
+      if (bi < 0) continue;
+      Block& o = s->blocks[bi];
+      if (o.staging) continue;             // (keeps an allocation of its own)
+      o.staging_row = Arena::round_up(o.nelem * j.grad_esize());
+      o.staging = j.stage_base + off;
+      o.staging_own = false;
+      off += o.staging_row * W;
+    }
+    if (b.staging) return PS_OK;
   }
-  // the staging buffer may still be read by the block's previous aggregate
-  ++s->call_id;
-  rc = order_after_block(s, *b, static_cast<cudaStream_t>(stream));
-  if (rc) return rc;
-  char* dst = static_cast<char*>(b->staging) + (size_t)worker * b->staging_row;
-  PS_CUDA(s, cudaMemcpyAsync(dst, host_ptr, b->nelem * j.grad_esize(), cudaMemcpyHostToDevice,
-                             static_cast<cudaStream_t>(stream)));
-  b->pushed[worker] = dst;
-  b->npushed++;
+  b.staging_row = Arena::round_up(b.nelem * j.grad_esize());
+  cudaError_t e = cudaMalloc(&b.staging, b.staging_row * W);
+  if (e != cudaSuccess) {
+    b.staging = nullptr;
+    cudaGetLastError();
+    if (e == cudaErrorMemoryAllocation) return PS_ERR_NOMEM;
+    s->cuda_err = cudaGetErrorString(e);
+    return PS_ERR_CUDA;
+  }
+  b.staging_own = true;
   return PS_OK;
+}
+
+int ps_push_host_batch(ps_service* s, int n, const int* jobs, const int* blocks, const int* workers,
+                       const void* const* host_ptrs, void* stream_) {
+  if (!alive(s)) return PS_ERR_BAD_HANDLE;
+  std::lock_guard<std::mutex> lk(s->mu);
+  if (n < 0 || (n > 0 && (!jobs || !blocks || !workers || !host_ptrs))) return PS_ERR_BAD_ARG;
+  // validation first: nothing is copied or recorded unless every entry is acceptable
+  std::vector<Block*> bs((size_t)n);
+  const unsigned long long gen = ++s->gen;
+  for (int i = 0; i < n; ++i) {
+    int rc = push_checked(s, jobs[i], blocks[i], workers[i], host_ptrs[i], &bs[i], false);
+    if (rc) return rc;
+  }
+  {                                        // the same (block, worker) twice in one batch
+    std::vector<unsigned char> seen;
+    for (int i = 0; i < n; ++i) {
+      Block& b = *bs[i];
+      if (b.mark != gen) { b.mark = gen; b.mark_pos = (int)seen.size(); seen.resize(seen.size() + b.pushed.size(), 0); }
+      unsigned char& f = seen[(size_t)b.mark_pos + (size_t)workers[i]];
+      if (f) return PS_ERR_DUPLICATE;
+      f = 1;
+    }
+  }
+  if (!has_device(s)) return PS_ERR_NO_DEVICE;
+  if (n == 0) return PS_OK;
+  PS_CUDA(s, cudaSetDevice(s->device));
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  for (int i = 0; i < n; ++i) {
+    int rc = ensure_staging(s, *bs[i]);
+    if (rc) return rc;
+  }
+  // the staging rows may still be read by the blocks' previous aggregates
+  ++s->call_id;
+  unsigned int waited = 0;
+  for (int i = 0; i < n; ++i) {
+    if (i && bs[i] == bs[i - 1]) continue;
+    int rc = order_after_block(s, *bs[i], stream, &waited);
+    if (rc) return rc;
+  }
+  // copies: neighbours on both sides are merged (the padding between rows travels with them)
+  struct Range { char* dst; const char* src; size_t bytes; size_t span; };
+  std::vector<Range> rs((size_t)n);
+  for (int i = 0; i < n; ++i) {
+    Block& b = *bs[i];
+    rs[i].dst = static_cast<char*>(b.staging) + (size_t)workers[i] * b.staging_row;
+    rs[i].src = static_cast<const char*>(host_ptrs[i]);
+    rs[i].bytes = b.nelem * s->jobs[b.job].grad_esize();
+    rs[i].span = b.staging_row;
+  }
+  std::vector<int> order((size_t)n);
+  for (int i = 0; i < n; ++i) order[i] = i;
+  std::sort(order.begin(), order.end(), [&](int a, int b) { return rs[a].dst < rs[b].dst; });
+  for (size_t k = 0; k < order.size();) {
+    const Range& first = rs[order[k]];
+    size_t len = first.bytes, span = first.span, m = k + 1;
+    while (m < order.size() && rs[order[m]].dst == first.dst + span && rs[order[m]].src == first.src + span) {
+      len = span + rs[order[m]].bytes;
+      span += rs[order[m]].span;
+      ++m;
+    }
+    PS_CUDA(s, cudaMemcpyAsync(first.dst, first.src, len, cudaMemcpyHostToDevice, stream));
+    k = m;
+  }
+  for (int i = 0; i < n; ++i) {
+    bs[i]->pushed[workers[i]] = rs[i].dst;
+    bs[i]->npushed++;
+  }
+  return PS_OK;
+}
+
+int ps_push_host(ps_service* s, int job, int block, int worker, const void* host_ptr, void* stream) {
+  return ps_push_host_batch(s, 1, &job, &block, &worker, &host_ptr, stream);
 }
 
 static int launch_plan(ps_service* s, const std::vector<int>& idx, Plan& plan, cudaStream_t stream,
@@ -1669,10 +1764,8 @@ int ps_unregister_block(ps_service* s, int job, int block) {
       if (rc) return rc;
       b.mig_batch = -1;
     }
-    if (b.staging) {
-      PS_CUDA(s, cudaFree(b.staging));
-      b.staging = nullptr;
-    }
+    if (b.staging && b.staging_own) PS_CUDA(s, cudaFree(b.staging));
+    b.staging = nullptr;                   // (a range of the job's region stays with the region)
   }
   s->ctxs[b.ctx].arena.release(b.off, b.bytes);
   s->jobs[b.job].block_of_id[b.id] = -1;

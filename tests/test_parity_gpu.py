@@ -261,3 +261,73 @@ def test_pinned_host_shards_are_read_in_place(opt, dt):
         pair.compare()
     finally:
         pair.close()
+
+
+@pytest.mark.parametrize("opt,dt", [(configs.SGD, configs.F32), (configs.ADAM, configs.BF16)])
+@pytest.mark.parametrize("layout", ["packed", "scattered"])
+def test_batched_pushes_from_host_memory(opt, dt, layout):
+    """ps_push_host_batch: shards in pinned host memory, either in the layout the
+    library sends as one copy (block after block, worker after worker, rows
+    padded to 256 bytes) or anywhere; three iterations reuse the staging region
+    while the previous aggregate may still be reading it; a block registered
+    after the region was allocated gets staging of its own."""
+    sizes = [70_001, 5, 4096, 12_345, 300_000]
+    cfg = tiny_config(sizes, 3, opt=opt, grad_dtype=dt)
+    pair = Pair(cfg)
+    svc = pair.svc
+    try:
+        job = cfg.jobs[0]
+        esz = 2 if dt == configs.BF16 else 4
+        rows = [(b.nelem * esz + 255) // 256 * 256 for b in job.blocks]
+        total = sum(r * job.num_workers for r in rows)
+        stream = torch.cuda.Stream()
+        every = configs.rounds_all(cfg)[0]
+        pools = []
+        for it in range(3):
+            slab = generate.grad_slab(cfg, 0, it)
+            host = to_np(slab)
+            raw = slab.contiguous().view(torch.uint8) if dt == configs.F32 else slab.contiguous().view(torch.int16).view(torch.uint8)
+            pool = torch.zeros(2 * total + 4096, dtype=torch.uint8).pin_memory()
+            pools.append(pool)                                   # stays alive until the copies have run
+            jobs, blocks, workers, ptrs = [], [], [], []
+            cur = 0
+            for b, row in zip(job.blocks, rows):
+                for w in range(job.num_workers):
+                    off = cur if layout == "packed" else 2 * total - cur - row + (16 if b.block % 2 else 0)
+                    n = b.nelem * esz
+                    pool[off:off + n].copy_(raw[w, b.job_offset * esz:b.job_offset * esz + n])
+                    jobs.append(0); blocks.append(b.block); workers.append(w); ptrs.append(pool.data_ptr() + off)
+                    pair.ora.push(0, b.block, w, host[w, b.job_offset:b.job_offset + b.nelem])
+                    cur += row
+            svc.push_host_batch(np.array(jobs, np.int32), np.array(blocks, np.int32), np.array(workers, np.int32),
+                                np.array(ptrs, np.uint64), stream)
+            pair.aggregate(every, stream)
+        # a (block, worker) twice in one batch, and a batch with one bad entry, change nothing
+        one = np.array([0], np.int32)
+        with pytest.raises(B.PsError) as e:
+            svc.push_host_batch(np.array([0, 0], np.int32), np.array([1, 1], np.int32), np.array([2, 2], np.int32),
+                                np.array([pools[0].data_ptr()] * 2, np.uint64), stream)
+        assert e.value.status == B.PS_ERR_DUPLICATE
+        with pytest.raises(B.PsError) as e:
+            svc.push_host_batch(np.array([0, 0], np.int32), np.array([1, 9], np.int32), np.array([0, 0], np.int32),
+                                np.array([pools[0].data_ptr()] * 2, np.uint64), stream)
+        assert e.value.status == B.PS_ERR_BAD_ARG
+        with pytest.raises(B.PsError) as e:
+            svc.aggregate([(0, 1)], stream)
+        assert e.value.status == B.PS_ERR_NOT_READY
+        # a block that did not exist when the job's staging region was laid out
+        late = torch.full((1000,), 0.25).pin_memory()
+        svc.register_block(0, 7, 1000, 0, None)
+        pair.ora.register_block(0, 7, 1000, 0, None)
+        ldata = late.to(torch.bfloat16) if dt == configs.BF16 else late
+        for w in range(job.num_workers):
+            svc.push_host_batch(one, np.array([7], np.int32), np.array([w], np.int32),
+                                np.array([ldata.data_ptr()], np.uint64), stream)
+            pair.ora.push(0, 7, w, to_np(ldata))
+        pair.aggregate([(0, 7)], stream)
+        stream.synchronize()
+        pair.compare()
+        n = 1000
+        assert np.array_equal(svc.view(svc.pull(0, 7), n).cpu().numpy(), pair.ora.pull(0, 7))
+    finally:
+        pair.close()
