@@ -111,13 +111,18 @@ enum {
                               block that waits in the batch, ...).  An idle device gets every round at
                               once.  Results are identical; what changes is how many launches carry
                               them.  0: one launch per round. */
+  PS_OPT_WAIT_CYCLES = 11, /* bulk-copy kernel: how many SM clock cycles a warp waits for a ring stage
+                              before it gives up, records the failure in the status word
+                              (ps_device_status) and lets the launch end; default 4e9 (about 2 s).
+                              Results of a launch that gave up are undefined. */
   PS_OPT_WORK_STREAMS = 9, /* with PS_OPT_OVERLAP: launches rotate over this many service-owned streams
                               (1..8, default 4) */
   PS_OPT_PROFILE = 5,      /* 1: aggregates record per-task device time (see ps_block_profile);
                               costs a few atomics per chunk; direct-load kernel only; default 0 */
   PS_OPT_KERNEL = 4        /* kernel variant: 0 = automatic (direct loads), 1 = direct loads,
-                              2 = bulk-copy ring; results are identical except for the
-                              rounding of the per-block norm */
+                              2 = bulk-copy ring (shards staged through shared memory by the TMA
+                              unit); results are identical except for the rounding of the
+                              per-block norm */
 };
 
 /* Creates an Aggregator service on GPU `device` with `num_contexts` contexts

@@ -188,6 +188,7 @@ struct ps_service {
   std::vector<int> batch;                  // block indices, in arrival order
   unsigned long long batch_chunks = 0;     // their size in chunks of kChunkAuto elements
   long long opt_batch = 1;
+  long long opt_wait_cycles = 4000000000ll;   // bulk-copy kernel: limit of a wait inside the kernel (about 2 s)
   bool mig_large_ok = true;                // the 28 KB kernel-parameter form of the migration kernel is accepted
   unsigned long long epoch = 0;            // bumped by whatever can invalidate a prepared round's table:
                                            // migration, import, unregistration, options
@@ -373,13 +374,9 @@ unsigned int auto_chunk(ps_service* s, const std::vector<int>& idx, int grid) {
   return ce;
 }
 
-// Elements per ring tile of the bulk-copy kernel: the largest multiple of 128
-// whose rows (W shards, parameters, state) fit one stage; 0 if none does.
-unsigned int tile_elems_for(const Job& j) {
-  const size_t in_bytes = (size_t)j.d.num_workers * j.grad_esize() + 4 * (1 + j.nstate());
-  const size_t t = (size_t)kStageBytes / in_bytes / kTileQuantum * kTileQuantum;
-  return (unsigned int)t;
-}
+// Elements per ring tile of the bulk-copy kernel (0 would mean: direct loads only).  A
+// tile is cut along the workers, so any number of workers fits.
+unsigned int tile_elems_for(const Job&) { return kRingTile; }
 
 // The fields of a task that change from one aggregate of its block to the next.
 void set_step_fields(const Job& j, const Block& b, PsTaskDev* t) {
@@ -497,6 +494,7 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
   h->profile = s->opt_profile ? 1u : 0u;
   h->sparse_off = (unsigned int)sparse_off;
   h->exited = 0;
+  h->wait_units = (unsigned int)std::min<long long>(0xffffffffll, (s->opt_wait_cycles + kWaitUnit - 1) / kWaitUnit);
   return PS_OK;
 }
 
@@ -1128,7 +1126,7 @@ static int launch_plan(ps_service* s, const std::vector<int>& idx, Plan& plan, c
     PS_CUDA(s, cudaStreamWaitEvent(run, sl->copied, 0));
     if (bulk)
       le = launch_kernel(ps_aggregate_bulk_kernel, grid, kBulkThreads, kBulkSmemBytes, run, false, sl->dev,
-                         (const PsJobDev*)s->jobs_dev, s->stats_dev, sl->partials, s->status_dev);
+                         (const PsJobDev*)s->jobs_dev, s->stats_dev, sl->partials, s->status_dev, done_word, seq);
     else
       le = launch_kernel(ps_aggregate_ldg_kernel, grid, kThreads, 0, run, false, sl->dev,
                          (const PsJobDev*)s->jobs_dev, s->stats_dev, sl->partials, done_word, seq);
@@ -1139,7 +1137,7 @@ static int launch_plan(ps_service* s, const std::vector<int>& idx, Plan& plan, c
     return PS_ERR_CUDA;
   }
   sl->seq = seq;
-  sl->signals = !bulk;
+  sl->signals = true;
   sl->stream = run;
   sl->work_stream = ws;
   sl->done_recorded = false;
@@ -1899,6 +1897,10 @@ int ps_set_option(ps_service* s, int option, long long value) {
     case PS_OPT_BATCH:
       s->opt_batch = value ? 1 : 0;
       return PS_OK;
+    case PS_OPT_WAIT_CYCLES:
+      if (value < 1) return PS_ERR_BAD_ARG;
+      s->opt_wait_cycles = value;
+      return PS_OK;
     case PS_OPT_WORK_STREAMS:
       if (value < 1 || value > kWorkStreams) return PS_ERR_BAD_ARG;
       s->opt_streams = value;
@@ -1924,6 +1926,7 @@ int ps_get_option(ps_service* s, int option, long long* out) {
     case PS_OPT_PDL: *out = s->opt_pdl; return PS_OK;
     case PS_OPT_WORK_STREAMS: *out = s->opt_streams; return PS_OK;
     case PS_OPT_BATCH: *out = s->opt_batch; return PS_OK;
+    case PS_OPT_WAIT_CYCLES: *out = s->opt_wait_cycles; return PS_OK;
     default: return PS_ERR_BAD_ARG;
   }
 }
@@ -2091,7 +2094,7 @@ __global__ void ps_noalloc_setup_kernel(NoAllocArgs a) {
     h.profile = 0;
     h.sparse_off = 0;
     h.exited = 0;
-    h._r2 = 0;
+    h.wait_units = 0;
     *reinterpret_cast<PsTableHdr*>(base) = h;
     *reinterpret_cast<PsTaskDev*>(base + kNaTaskOff) = a.task;     // ticket = 0 inside
     *reinterpret_cast<unsigned int*>(base + kNaStartsOff) = 0;

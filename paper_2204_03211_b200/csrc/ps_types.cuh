@@ -57,7 +57,7 @@ struct __align__(16) PsTableHdr {      // 48 bytes at the start of the table
   unsigned int profile;                // 1: record per-task device time (direct-load kernel)
   unsigned int sparse_off;             // byte offset of the PsSparseDev array (row-sparse shards)
   unsigned int exited;                 // CTAs that have left the launch (uploaded as 0)
-  unsigned int _r2;
+  unsigned int wait_units;             // bulk-copy kernel: limit of every mbarrier wait, in units of 1024 cycles
 };
 
 // One worker's shard of a row-sparse task: the sorted ids of the rows it holds

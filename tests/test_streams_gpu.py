@@ -180,3 +180,42 @@ def test_batched_migration_is_all_or_nothing_and_chains_without_host_waits():
             tiny.close()
     finally:
         pair.close()
+
+
+def test_ring_kernel_gives_up_when_its_wait_limit_runs_out_and_says_so():
+    """Every wait inside the bulk-copy kernel is bounded.  With the limit set to
+    about a thousand cycles — less than one round trip to HBM — the first
+    consumer wait of an otherwise ordinary launch runs out: the kernel records
+    it in the status word, lets its copies in flight land and returns promptly;
+    the context stays usable and a launch with the default limit on freshly
+    registered blocks matches the oracle bit for bit."""
+    import time
+    cfg = tiny_config([1 << 22] * 4, 8)
+    pair = Pair(cfg, kernel=2)
+    try:
+        pair.svc.set_option(B.PS_OPT_WAIT_CYCLES, 64)
+        assert pair.svc.get_option(B.PS_OPT_WAIT_CYCLES) == 64
+        pair.push_iteration(0)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        pair.svc.aggregate(configs.rounds_all(cfg)[0])
+        status = pair.svc.device_status()                # waits for the device
+        assert time.perf_counter() - t0 < 5.0            # no wait inside the kernel outlived its limit by much
+        assert status != 0
+        assert pair.svc.launch_info()["kernel"] == "bulk"
+        with pytest.raises(B.PsError):
+            pair.svc.set_option(B.PS_OPT_WAIT_CYCLES, 0)
+    finally:
+        pair.close()
+    x = torch.ones(1 << 20, device="cuda")               # the context is healthy
+    assert float(x.sum()) == float(1 << 20)
+    again = Pair(cfg, kernel=2)                          # default limit, fresh blocks
+    try:
+        for it in range(2):
+            again.push_iteration(it)
+            again.aggregate(configs.rounds_all(cfg)[0])
+        assert again.svc.device_status() == 0
+        assert again.svc.launch_info()["kernel"] == "bulk"
+        again.compare()
+    finally:
+        again.close()
