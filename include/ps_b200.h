@@ -87,10 +87,13 @@ enum {
                               gradient buffers or reads results on its own streams; ps_pull_host,
                               ps_block_stats, ps_block_profile, ps_migrate_block and ps_push_host
                               order themselves after the block's last launch in either mode.
-                              A launch that must follow an unfinished one (a block aggregated again)
-                              goes to that launch's stream; completion is learnt from a word each
-                              kernel stores to page-locked host memory, so a launch costs no event
-                              unless another stream has to wait for it.
+                              A small launch that must follow an unfinished one (a block aggregated
+                              again) goes to that launch's stream, where stream order is the
+                              dependency; large launches rotate over the service's streams and wait
+                              for exactly the launches they depend on.  What only the host has to
+                              know (may a table slot be reused, has a block's last launch finished,
+                              how many launches are running) it reads from a word that the last CTA
+                              of every launch stores to page-locked host memory.
                               Default 0: every launch is enqueued on `stream` itself. */
   PS_OPT_INLINE_TABLE = 7, /* 1 (default): a launch whose task table fits 3968 bytes (a round of a few
                               tensors) and has few chunks passes the table as a kernel parameter, one

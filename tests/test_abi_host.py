@@ -185,6 +185,19 @@ def test_options_validate():
     assert _status(s.set_option, 99, 1) == B.PS_ERR_BAD_ARG
     s.set_option(B.PS_OPT_CTAS_PER_SM, 2)
     assert s.get_option(B.PS_OPT_CTAS_PER_SM) == 2 and s.get_option(B.PS_OPT_SORT_TASKS) == 1
+    # defaults of the launch machinery, and their ranges
+    assert s.get_option(B.PS_OPT_BATCH) == 1 and s.get_option(B.PS_OPT_PDL) == 1
+    assert s.get_option(B.PS_OPT_WORK_STREAMS) == 4 and s.get_option(B.PS_OPT_WAIT_CYCLES) == 4_000_000_000
+    assert _status(s.set_option, B.PS_OPT_WORK_STREAMS, 0) == B.PS_ERR_BAD_ARG
+    assert _status(s.set_option, B.PS_OPT_WORK_STREAMS, 9) == B.PS_ERR_BAD_ARG
+    assert _status(s.set_option, B.PS_OPT_WAIT_CYCLES, 0) == B.PS_ERR_BAD_ARG
+    s.set_option(B.PS_OPT_WORK_STREAMS, 8)
+    s.set_option(B.PS_OPT_BATCH, 0)
+    assert s.get_option(B.PS_OPT_WORK_STREAMS) == 8 and s.get_option(B.PS_OPT_BATCH) == 0
+    # nothing is ever held back on a service without a device: flush and join are no-ops
+    s.flush()
+    s.join(None)
+    assert [v["launches"] for v in s.launch_stats()] == [0, 0, 0]
 
 
 def test_arena_accounting_and_exhaustion():
