@@ -202,8 +202,9 @@ int ps_push_batch(ps_service* svc, int n, const int* jobs, const int* blocks, co
                   const void* const* grad_dev_ptrs);
 
 /* Push from host memory: copies nelem gradient values from `grad_host_ptr`
- * into a service-owned device staging buffer (allocated on first use for this
- * block) with cudaMemcpyAsync on `stream`, then records the push.  The host
+ * into a service-owned device staging buffer (allocated at the job's first push
+ * from host memory, see ps_push_host_batch) with cudaMemcpyAsync on `stream`,
+ * then records the push.  The host
  * buffer must stay valid until that copy completes; the ps_aggregate that
  * consumes the push must be enqueued on the same stream (or one ordered after
  * it).  Errors as ps_push, plus NOMEM, CUDA, NO_DEVICE. */

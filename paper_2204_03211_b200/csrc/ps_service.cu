@@ -569,7 +569,6 @@ int acquire_slot(ps_service* s, size_t table_bytes, size_t nchunks, Slot** out) 
     PS_CUDA(s, cudaMemset(sl.mut, 0, kInlineMaxTasks * sizeof(PsTaskMut)));   // kept all-zero by the kernel
     PS_CUDA(s, cudaStreamSynchronize(cudaStreamLegacy));                      // before a service stream uses it
   }
-  sl.gen = s->gen;
   *out = &sl;
   return PS_OK;
 }
@@ -1137,6 +1136,7 @@ static int launch_plan(ps_service* s, const std::vector<int>& idx, Plan& plan, c
     return PS_ERR_CUDA;
   }
   sl->seq = seq;
+  sl->gen = seq;                           // what a block remembers of its last launch (unique per launch)
   sl->signals = true;
   sl->stream = run;
   sl->work_stream = ws;
