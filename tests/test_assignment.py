@@ -245,3 +245,28 @@ def test_planner_argument_errors(_lib):
     t, n = p.assign(j, 2.5)
     assert p.task_info(t) == (j, n, 2.5)
     assert p.remove_job(j) == 1 and status(p.task_info, t) == B.PS_ERR_BAD_ARG
+
+
+def test_planner_under_address_and_undefined_behaviour_sanitizers(tmp_path):
+    """The host-only planner, built from source with -fsanitize=address,undefined
+    together with a C++ driver that runs six long seeded sequences of arrivals,
+    assignments and exits: an out-of-bounds access, a use after free, a leak or
+    undefined arithmetic aborts the run.  (The device code cannot be run under a
+    sanitizer here; what guards it is the element-wise comparison with the
+    oracle and the zero-padding checks.)"""
+    import shutil
+    import subprocess
+    if shutil.which("g++") is None:
+        pytest.skip("no g++")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    exe = str(tmp_path / "planner_sanitized")
+    cmd = ["g++", "-std=c++17", "-O1", "-g", "-fsanitize=address,undefined", "-fno-sanitize-recover=all",
+           "-I", os.path.join(root, "include"), "-o", exe, os.path.join(root, "tests", "c", "planner_sanitized.cpp"),
+           os.path.join(root, "paper_2204_03211_b200", "csrc", "ps_planner.cpp")]
+    built = subprocess.run(cmd, capture_output=True, text=True)
+    if built.returncode != 0 and ("asan" in built.stderr or "ubsan" in built.stderr or "sanitize" in built.stderr):
+        pytest.skip("sanitizer runtime not installed")
+    assert built.returncode == 0, built.stderr[-2000:]
+    r = subprocess.run([exe], capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, (r.stdout + r.stderr)[-3000:]
+    assert "planner_sanitized: ok" in r.stdout
