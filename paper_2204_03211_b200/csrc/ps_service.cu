@@ -262,8 +262,10 @@ int reap_frees(ps_service* s, bool wait) {
   return PS_OK;
 }
 
-int arena_alloc(ps_service* s, int ctx, size_t bytes, size_t* off_out) {
-  if (has_device(s)) {
+// reap = false: the caller has just released what finished migrations left behind (a batch of
+// many blocks does that once, not once per block: the list it walks is as long as the batch)
+int arena_alloc(ps_service* s, int ctx, size_t bytes, size_t* off_out, bool reap = true) {
+  if (reap && has_device(s)) {
     int rc = reap_frees(s, false);
     if (rc) return rc;
   }
@@ -1563,11 +1565,15 @@ static int free_batch(ps_service* s, int* out) {
 static int migrate_many(ps_service* s, const std::vector<int>& bis, int dst_ctx, cudaStream_t stream) {
   struct Move { int bi; size_t noff; };
   std::vector<Move> moves;
+  {
+    int rc = reap_frees(s, false);
+    if (rc) return rc;
+  }
   for (int bi : bis) {
     Block& b = s->blocks[bi];
     if (b.ctx == dst_ctx) continue;
     size_t noff = 0;
-    int rc = arena_alloc(s, dst_ctx, b.bytes, &noff);
+    int rc = arena_alloc(s, dst_ctx, b.bytes, &noff, false);
     if (rc) {
       for (auto& m : moves) s->ctxs[dst_ctx].arena.release(m.noff, s->blocks[m.bi].bytes);
       return rc;
