@@ -634,6 +634,7 @@ def main():
     ap.add_argument("--in-stream", action="store_true",
                     help="enqueue every launch on the caller's stream (PS_OPT_OVERLAP = 0) instead of letting "
                          "the launches of a step overlap on the service's streams and joining once per step")
+    ap.add_argument("--no-split", action="store_true", help="PS_OPT_SPLIT = 0: a large set of ready blocks is one launch")
     ap.add_argument("--no-batch", action="store_true", help="PS_OPT_BATCH = 0: one launch per round, never packed")
     ap.add_argument("--streams", type=int, default=0, help="PS_OPT_WORK_STREAMS (0 = the library's default)")
     ap.add_argument("--unprepared", action="store_true",
@@ -740,6 +741,7 @@ def main():
     wl.svc.set_option(B.PS_OPT_KERNEL, args.kernel)
     wl.svc.set_option(B.PS_OPT_PDL, int(not args.no_pdl))
     wl.svc.set_option(B.PS_OPT_BATCH, int(not args.no_batch))
+    wl.svc.set_option(B.PS_OPT_SPLIT, int(not args.no_split))
     if args.streams:
         wl.svc.set_option(B.PS_OPT_WORK_STREAMS, args.streams)
     wl.overlap = not args.in_stream

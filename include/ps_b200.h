@@ -114,6 +114,11 @@ enum {
                               block that waits in the batch, ...).  An idle device gets every round at
                               once.  Results are identical; what changes is how many launches carry
                               them.  0: one launch per round. */
+  PS_OPT_SPLIT = 12,       /* 1 (default), with PS_OPT_OVERLAP and PS_OPT_BATCH for rounds given with
+                              PS_ROUND_INPUTS_COMPLETE: a set of ready blocks that fills several waves
+                              of CTAs is sent as up to four consecutive launches of at least a wave and
+                              a half each, on different streams, so that the tail of one overlaps the
+                              start of the next.  0: one launch.  Same results. */
   PS_OPT_WAIT_CYCLES = 11, /* bulk-copy kernel: how many SM clock cycles a warp waits for a ring stage
                               before it gives up, records the failure in the status word
                               (ps_device_status) and lets the launch end; default 4e9 (about 2 s).

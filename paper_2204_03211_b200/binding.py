@@ -31,6 +31,7 @@ PS_OPT_PDL = 8
 PS_OPT_WORK_STREAMS = 9
 PS_OPT_BATCH = 10
 PS_OPT_WAIT_CYCLES = 11
+PS_OPT_SPLIT = 12
 PS_ROUND_INPUTS_COMPLETE = 1
 
 

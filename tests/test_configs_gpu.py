@@ -84,10 +84,11 @@ def test_c4_twelve_packed_jobs_bursty_arrival_every_element(overlap):
             pair.iteration(it, rounds)
             if it in (0, cfg.iterations - 1):
                 assert pair.compare(it + 1) == cfg.num_params
-        # one more iteration with everything ready at once: a single packed launch
+        # one more iteration with everything ready at once: a single packed round
         before = pair.svc.launch_info()["launches"]
         pair.iteration(cfg.iterations, configs.rounds_all(cfg))
-        assert pair.svc.launch_info()["launches"] == before + 1
+        # in the caller's stream: one launch; overlapped: up to four, whose tails and heads overlap
+        assert before + 1 <= pair.svc.launch_info()["launches"] <= before + (4 if overlap else 1)
         pair.compare(cfg.iterations + 1)
     finally:
         pair.close()

@@ -119,6 +119,7 @@ def test_small_and_large_launches_interleave():
     svc = pair.svc
     try:
         svc.set_option(B.PS_OPT_OVERLAP, 1)
+        svc.set_option(B.PS_OPT_SPLIT, 0)         # one launch per round: split, the large round's parts would fit the parameters too
         every = configs.rounds_all(cfg)[0]
         small = [t for t in every if cfg.jobs[0].blocks[t[1]].nelem <= 3000]
         big = [t for t in every if t not in small]
