@@ -13,6 +13,13 @@ blocks it touches.  Reported per model:
   exposed_ms  extra time of "aggregate, migrate everything, aggregate again"
               over "aggregate, aggregate" — the part of the move the job sees
               when the next update follows immediately (no idle window to hide it)
+  chain_ms    device time per move when three moves (there, back, there) are
+              enqueued back to back: the host part of call k+1 (reserving the
+              destination ranges, building the range table) runs while the copy
+              of call k is still on the device, as it does when several jobs'
+              models move in a row; copy_ms is the cold case, one call on an
+              idle stream, host part included
+  host_ms     host time inside one ps_migrate_blocks call
   hidden_ms   extra time of the first aggregate AFTER a completed move over an
               ordinary aggregate (the paper's case: the window between the last
               Pull and the next Update hides the copy) — expected about zero
@@ -25,6 +32,7 @@ import argparse
 import json
 import os
 import sys
+import time
 
 import numpy as np
 import torch
@@ -41,7 +49,9 @@ def one_model(model: str, workers: int, reps: int, one_by_one: bool = False):
     job = configs._job(model, model, workers, lr=0.1, momentum=0.9, weight_decay=1e-4)
     cfg = configs.Config("mig-" + model, 7, 1, [job], num_contexts=2)
     dev = torch.device("cuda", 0)
-    arena = sum(2 * (4 * b.nelem + 256) for b in job.blocks) + (64 << 20)
+    # room for the model twice per context: in a chain of moves the ranges a block left are
+    # released only once its copy has completed
+    arena = 2 * sum(2 * (4 * b.nelem + 256) for b in job.blocks) + (64 << 20)
     svc = B.Service(0, 2, arena)
     j = svc.register_job(**job.hparams())
     p0 = generate.init_params(cfg, 0, dev)
@@ -86,7 +96,7 @@ def one_model(model: str, workers: int, reps: int, one_by_one: bool = False):
         aggregate()
         migrate_all(flip())
     torch.cuda.synchronize()
-    base, exposed, hidden, copy, single = [], [], [], [], []
+    base, exposed, hidden, copy, single, chain, host = [], [], [], [], [], [], []
     for _ in range(reps):
         base.append(timed(lambda: (aggregate(), aggregate())))
         exposed.append(timed(lambda: (aggregate(), migrate_all(flip()), aggregate())))
@@ -104,10 +114,20 @@ def one_model(model: str, workers: int, reps: int, one_by_one: bool = False):
         e1.record(side)
         torch.cuda.synchronize()
         copy.append(e0.elapsed_time(e1))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(side)
+        t0 = time.perf_counter()
+        for _ in range(3):                  # (a fourth would wait for the first: the arenas hold the model twice)
+            migrate_all(flip())
+        host.append((time.perf_counter() - t0) * 1e3 / 3)
+        e1.record(side)
+        torch.cuda.synchronize()
+        chain.append(e0.elapsed_time(e1) / 3)
     med = lambda v: float(sorted(v)[len(v) // 2])
     moved = sum(2 * ((4 * b.nelem + 255) // 256 * 256) for b in job.blocks)
     out = {"model": model, "params": job.num_params, "blocks": len(job.blocks), "workers": workers,
            "calls": "one ps_migrate_block per block" if one_by_one else "one ps_migrate_blocks", "bytes_moved": moved, "copy_ms": med(copy), "copy_gbs": 2 * moved / med(copy) / 1e6,
+           "chain_ms": med(chain), "chain_gbs": 2 * moved / med(chain) / 1e6, "host_ms": med(host),
            "two_aggregates_ms": med(base), "exposed_ms": med(exposed) - med(base),
            "one_aggregate_ms": med(single), "hidden_ms": med(hidden) - med(single)}
     svc.close()

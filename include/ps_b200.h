@@ -300,8 +300,8 @@ int ps_migrate_block(ps_service* svc, int job, int block, int dst_ctx, void* str
 /* The same for n blocks at once (host array of tasks, no block listed twice), as
  * ONE batch: every destination range is reserved first (PS_ERR_NOMEM leaves all
  * blocks where they were), one gather-copy kernel moves up to 1024 blocks (96
- * where the driver refuses a 28 KB parameter block) and one event marks the
- * batch — moving all tensors of a model costs one launch instead of one copy
+ * where the driver refuses a parameter block above 4 KB) and one event marks
+ * the batch — moving all tensors of a model costs one launch instead of one copy
  * call per tensor (the paper's Appendix B measures
  * exactly that case: the overhead of migrating all tensors of a model).
  * Errors: BAD_ARG, DUPLICATE, NOMEM, NO_DEVICE, CUDA. */

@@ -4,20 +4,22 @@
 // metadata, here the optimizer state — to the new one).  Ranges are 256-byte
 // aligned and a multiple of 256 bytes long (arena granularity); work is cut
 // into 64 KB tiles that CTAs take round-robin.  The range table travels as a
-// kernel parameter: 96 ranges fit the 4 KB every driver accepts; the 1024-range
-// form (28 KB) uses the large parameter space of current drivers, so that all
-// blocks of a model move in one launch with no gap in the middle.
+// kernel parameter: 96 ranges fit the 4 KB every driver accepts; the 256- and
+// 1024-range forms (7 and 28 KB) use the large parameter space of current
+// drivers, so that all blocks of a model move in one launch with no gap in the
+// middle.
 #pragma once
 
 #include <cuda_runtime.h>
 
 namespace psb {
 
-constexpr int kMigSmall = 96, kMigLarge = 1024;
+constexpr int kMigSmall = 96, kMigMedium = 256, kMigLarge = 1024;
 constexpr unsigned int kMigTile = 65536;
 
 template <int N>
 struct MigArgs {                       // passed by value
+  static constexpr int kRanges = N;
   const unsigned char* src[N];
   unsigned char* dst[N];
   unsigned long long bytes[N];

@@ -14,6 +14,7 @@
 #include <algorithm>
 #include <chrono>
 #include <thread>
+#include <type_traits>
 #include <cmath>
 #include <cstdint>
 #include <cstdio>
@@ -1673,15 +1674,28 @@ static int migrate_many(ps_service* s, const std::vector<int>& bis, int dst_ctx,
       args->tile_prefix[count] = tiles;
       return (int)std::min<unsigned int>(tiles, (unsigned int)s->num_sms * 16u);
     };
+    // the cost of a launch grows with its parameter bytes (measured: 21 us of host time
+    // with the 28 KB table), so the smallest table that holds what is left is taken
+    auto launch_as = [&](auto* args, size_t first, size_t count) {
+      using A = std::remove_pointer_t<decltype(args)>;
+      const int grid = launch_some(args, first, count);
+      ps_migrate_kernel<A::kRanges><<<grid, 256, 0, stream>>>(*args);
+      return cudaGetLastError();
+    };
     size_t first = 0;
     while (first < moves.size() && e == cudaSuccess) {
       const size_t left = moves.size() - first;
       if (left > (size_t)kMigSmall && s->mig_large_ok) {
-        static thread_local MigArgs<kMigLarge> big;
-        const size_t count = std::min<size_t>(kMigLarge, left);
-        const int grid = launch_some(&big, first, count);
-        ps_migrate_kernel<kMigLarge><<<grid, 256, 0, stream>>>(big);
-        e = cudaGetLastError();
+        size_t count = 0;
+        if (left <= (size_t)kMigMedium) {
+          static thread_local MigArgs<kMigMedium> mid;
+          count = left;
+          e = launch_as(&mid, first, count);
+        } else {
+          static thread_local MigArgs<kMigLarge> big;
+          count = std::min<size_t>(kMigLarge, left);
+          e = launch_as(&big, first, count);
+        }
         if (e != cudaSuccess) {            // refused at launch: nothing ran; remember and take the small form
           s->mig_large_ok = false;
           e = cudaSuccess;
@@ -1691,9 +1705,7 @@ static int migrate_many(ps_service* s, const std::vector<int>& bis, int dst_ctx,
       } else {
         MigArgs<kMigSmall> small;
         const size_t count = std::min<size_t>(kMigSmall, left);
-        const int grid = launch_some(&small, first, count);
-        ps_migrate_kernel<kMigSmall><<<grid, 256, 0, stream>>>(small);
-        e = cudaGetLastError();
+        e = launch_as(&small, first, count);
         first += count;
       }
     }
