@@ -128,6 +128,62 @@ def test_bf16_every_bit_pattern_sums_like_the_oracle(opt):
         pair.close()
 
 
+@pytest.mark.parametrize("opt", [configs.SGD, configs.ADAM])
+@pytest.mark.parametrize("kernel", [1, 2, 3], ids=["ldg", "bulk", "inline"])
+@pytest.mark.parametrize("shift", [0, 1], ids=["vector", "scalar"])
+def test_fp32_special_values_travel_like_ieee_binary32(opt, kernel, shift):
+    """No flush to zero, no fast division or root, no special cases: gradients
+    drawn from ALL binary32 bit patterns (subnormals, huge values that overflow
+    the sum, infinities, NaNs, sums that cancel to a signed zero) leave the
+    same bits in p and the state as the oracle's plain IEEE arithmetic, over
+    two iterations (the second consumes the state the first one left).  NaN
+    payloads are not compared: where the oracle has a NaN the kernel has one."""
+    W, n = 3, (1 << 18) + 37
+    # (no weight decay: wd * p would bury a subnormal aggregate, and with it a flushed one)
+    cfg = tiny_config([n], W, opt=opt, weight_decay=0.0)
+    pair = Pair(cfg, kernel=kernel)
+    try:
+        rng = np.random.default_rng(2204)
+        q = n // 4
+        s0 = rng.integers(0, 1 << 32, n, dtype=np.uint64).astype(np.uint32)
+        s1 = rng.integers(0, 1 << 32, n, dtype=np.uint64).astype(np.uint32)
+        s1[:q] &= 0x807FFFFF                                   # subnormal or zero
+        s1[q:2 * q] = (s1[q:2 * q] & 0x807FFFFF) | 0x7F000000  # about 1e38: sums overflow
+        s1[2 * q:3 * q] = s0[2 * q:3 * q] ^ 0x80000000         # the negative of worker 0: cancels
+        s1[3 * q::3] = 0x7F800000                              # +inf
+        s1[3 * q + 1::3] = 0xFF800000                          # -inf
+        s2 = rng.integers(0, 1 << 23, n, dtype=np.uint64).astype(np.uint32)    # positive subnormals
+        s2[1::2] |= 0x80000000
+        s2[2 * q:3 * q:2] = 0                                  # +0 after a cancelled sum
+        shards = [s0.view(np.float32), s1.view(np.float32), s2.view(np.float32)]
+        keep = []
+        for w, a in enumerate(shards):
+            buf = torch.empty(n + 4, dtype=torch.float32, device="cuda")
+            buf[shift:shift + n].copy_(torch.from_numpy(a.copy()))
+            keep.append(buf)
+        for it in range(2):
+            for w, a in enumerate(shards):
+                pair.svc.push(0, 0, w, keep[w].data_ptr() + 4 * shift)
+                pair.ora.push(0, 0, w, a)
+            if it == 0:
+                assert all(c.vector_path == (0 if shift else 1) for c in pair.svc.plan([(0, 0)]))
+            pair.aggregate([(0, 0)])
+            p, a, v, _ = pair.gpu_block(0, 0)
+            rp = pair.ora.pull(0, 0)
+            ra, rv = pair.ora.state(0, 0)
+            for name, got, ref in (("p", p, rp), ("state0", a, ra)) + ((("state1", v, rv),) if rv is not None else ()):
+                nan = np.isnan(ref)
+                assert np.array_equal(np.isnan(got), nan), "%s, iteration %d: NaN positions" % (name, it + 1)
+                assert np.array_equal(got[~nan].view(np.uint32), ref[~nan].view(np.uint32)), \
+                    "%s, iteration %d: bits" % (name, it + 1)
+            # the case has teeth: the state holds NaNs, infinities and non-zero subnormals
+            tiny = np.finfo(np.float32).tiny
+            assert np.isfinite(ra).sum() > n // 3 and np.isnan(ra).any() and (it > 0 or np.isinf(ra).any())
+            assert ((ra != 0) & (np.abs(ra) < tiny)).sum() > 100
+    finally:
+        pair.close()
+
+
 def test_small_rounds_travel_as_kernel_parameters_and_slots_stay_clean():
     """A round whose table fits the kernel-parameter limit launches without an
     upload.  Tasks of several chunks count their chunks in per-slot device
