@@ -118,7 +118,8 @@ enum {
                               PS_ROUND_INPUTS_COMPLETE: a set of ready blocks that fills several waves
                               of CTAs is sent as up to four consecutive launches of at least a wave and
                               a half each, on different streams, so that the tail of one overlaps the
-                              start of the next.  0: one launch.  Same results. */
+                              start of the next.  Only a single round is cut this way; what was packed
+                              from several rounds goes out as one launch.  0: one launch.  Same results. */
   PS_OPT_WAIT_CYCLES = 11, /* bulk-copy kernel: how many SM clock cycles a warp waits for a ring stage
                               before it gives up, records the failure in the status word
                               (ps_device_status) and lets the launch end; default 4e9 (about 2 s).
