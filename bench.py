@@ -38,15 +38,22 @@ METRIC = "aggregated_params_per_sec"
 UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of the dominant kernel from the committed ncu capture
-# (profiles/), as measured dram bytes per algorithmic byte, keyed by the hash
-# of the kernel source it was taken from.  A changed kernel reports null.
-NCU_TRAFFIC = {"kernel_sha": "4733ace9e33e", "dram_bytes_per_algorithmic_byte": 0.980}
+# DRAM traffic of the dominant kernel from the committed ncu captures
+# (profiles/), as measured dram bytes per algorithmic byte, per kernel, keyed by
+# the hash of the kernel source it was taken from.  A changed kernel (or one
+# without a capture) reports null.
+_SHARED_SOURCES = ("ps_types.cuh", "ps_math.cuh", "ps_rows.cuh")
+NCU_TRAFFIC = {
+    "ps_aggregate_ldg_kernel": {"sources": _SHARED_SOURCES + ("ps_kernel_ldg.cuh",), "kernel_sha": "4733ace9e33e",
+                                "dram_bytes_per_algorithmic_byte": 0.980},
+    "ps_aggregate_bulk_kernel": {"sources": _SHARED_SOURCES + ("ps_kernel_bulk.cuh",), "kernel_sha": "71fa71c736ea",
+                                 "dram_bytes_per_algorithmic_byte": 0.984},
+}
 
 
-def kernel_sha() -> str:
+def kernel_sha(kernel: str = "ps_aggregate_ldg_kernel") -> str:
     h = hashlib.sha256()
-    for name in ("ps_types.cuh", "ps_math.cuh", "ps_rows.cuh", "ps_kernel_ldg.cuh"):
+    for name in NCU_TRAFFIC.get(kernel, NCU_TRAFFIC["ps_aggregate_ldg_kernel"])["sources"]:
         with open(os.path.join(ROOT, "paper_2204_03211_b200", "csrc", name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:12]
@@ -779,10 +786,11 @@ def main():
     # the dominant kernel's average launch duration: the timed region's device time, less nothing —
     # its launches fill the region (other variants' byte share is printed beside it)
     dom_ms = sum(blocks) * dominant.get("byte_share", 1.0) / max(dominant["launches"], 1)
-    sha = kernel_sha()
+    sha = kernel_sha(dominant["kernel"])
     traffic = None
-    if NCU_TRAFFIC["kernel_sha"] == sha and NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"]:
-        traffic = per_launch_bytes * NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"]
+    captured = NCU_TRAFFIC.get(dominant["kernel"])
+    if captured and captured["kernel_sha"] == sha:
+        traffic = per_launch_bytes * captured["dram_bytes_per_algorithmic_byte"]
 
     e2e = e2e_mapped = None
     if not args.no_e2e:

@@ -1,17 +1,22 @@
 // Aggregation kernel, bulk-copy variant for sm_100a: one persistent CTA per SM,
 // warp-specialised.  A producer warp claims (job, block, chunk) work items from
-// the table's atomic counter, cuts each chunk into tiles of 2048 elements and
+// the table's atomic counter, cuts each chunk into tiles of 4096 elements and
 // streams every tile into a shared-memory ring with 1-D bulk asynchronous
 // copies (TMA unit, completion counted on an mbarrier; every CTA fetches its own
 // tiles, no multicast).  A tile is cut ALONG THE WORKERS: one ring stage holds
-// the tile's rows of a few consecutive workers (four fp32 or eight bf16 shards,
-// 8 KB or 4 KB per row, so every copy is large), the next stage the next
+// the tile's rows of a few consecutive workers (three fp32 or six bf16 shards,
+// 16 KB or 8 KB per row: issuing a copy costs the producer about a hundred
+// cycles whatever its size, so copies are made large), the next stage the next
 // workers, and the parameters and optimizer state ride in the tile's last
 // stage.  Eight consumer warps keep the running sums of a tile in registers
 // across its stages — worker order 0..W-1, binary32, so the bits are those of
 // the direct-load kernel — and on the last stage apply the optimizer and store
 // parameters and state with 128-bit stores.  The ring keeps 192 KB per SM in
-// flight whatever W is.
+// flight whatever W is.  A tenth warp collects each finished chunk's partial
+// sums of squares and draws the tickets that count a task's chunks when the
+// CTA has run out of work: done by the producer, per chunk, those round trips
+// to memory and their fences were the kernel's bottleneck — the producer has
+// about a thousand cycles per stage to keep the ring full.
 //
 // Chunks that cannot use bulk copies (a shard pointer that is not 16-byte
 // aligned, fewer elements than one vector) are handed to the consumers as
@@ -28,11 +33,14 @@ namespace psb {
 
 constexpr int kBulkConsumerWarps = 8;
 constexpr int kBulkConsumers = kBulkConsumerWarps * 32;     // 256 consumer threads
-constexpr int kBulkThreads = kBulkConsumers + 32;           // + one producer warp
-constexpr int kStageBytes = 32768;
-constexpr int kStages = 6;
+constexpr int kBulkThreads = kBulkConsumers + 64;           // + one producer warp + one publisher warp
+constexpr int kPubSlots = 8;                                // finished chunks waiting for the publisher
+constexpr unsigned int kPubEnd = 0xffffffffu;               // in place of a task: no more chunks from this CTA
+constexpr int kPubRuns = 8;                                 // chunks a CTA collects before it draws their tasks' tickets
+constexpr int kStageBytes = 49152;
+constexpr int kStages = 4;
 constexpr int kBulkSmemBytes = kStages * kStageBytes + 1024;
-constexpr unsigned int kRingTile = 2048;                    // elements per tile: 8 per consumer thread
+constexpr unsigned int kRingTile = 4096;                    // elements per tile: 16 per consumer thread
 constexpr long long kDrainCycles = 4000000000ll;            // limit of the producer's own wait for its copies (about 2 s)
 constexpr unsigned int kWaitUnit = 1024;                    // the table gives its wait limit in units of this many cycles
 
@@ -50,6 +58,7 @@ struct StageMeta {
   unsigned int nrows;                  // shard rows in this stage
   unsigned int state_off;              // byte offset of the p row (kTileLast), rows of kRingTile floats follow
   unsigned int flags;
+  unsigned int pub_slot;               // kChunkEnd: where the chunk's partial sums go
   int W, kind;                         // kind = (optimizer << 1) | gradient type
   Hp h;
 };
@@ -112,46 +121,51 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, unsigned in
 
 // ---- consumer bodies ------------------------------------------------------------
 
-// Adds the stage's shard rows to the thread's running sums.  fp32: the thread owns
-// the float4 groups c and c + 256 of the tile; bf16: the 8 elements of group c.
+// Adds the stage's shard rows to the thread's running sums.  A thread owns the
+// 16-byte groups c, c + 256, ... of every row: four groups of four fp32 elements,
+// or two groups of eight bf16 elements — 16 elements of the tile either way.
 template <bool BF16>
 __device__ __forceinline__ void ring_accumulate(unsigned int c, const unsigned char* __restrict__ st, unsigned int nrows,
-                                                unsigned int cnt, bool first, float (&acc)[8]) {
-  if (!BF16) {
-    const unsigned int ng = cnt >> 2;
-    const bool a0 = c < ng, a1 = c + kBulkConsumers < ng;
-    constexpr unsigned int kRow = kRingTile * 4;
-#pragma unroll 4
-    for (unsigned int r = 0; r < nrows; ++r) {
-      const uint4* row = reinterpret_cast<const uint4*>(st + (size_t)r * kRow);
-      uint4 x0 = make_uint4(0, 0, 0, 0), x1 = x0;
-      if (a0) x0 = row[c];
-      if (a1) x1 = row[c + kBulkConsumers];
-      if (first && r == 0) {
-        acc[0] = __uint_as_float(x0.x); acc[1] = __uint_as_float(x0.y); acc[2] = __uint_as_float(x0.z); acc[3] = __uint_as_float(x0.w);
-        acc[4] = __uint_as_float(x1.x); acc[5] = __uint_as_float(x1.y); acc[6] = __uint_as_float(x1.z); acc[7] = __uint_as_float(x1.w);
-      } else {
-        acc[0] = __fadd_rn(acc[0], __uint_as_float(x0.x)); acc[1] = __fadd_rn(acc[1], __uint_as_float(x0.y));
-        acc[2] = __fadd_rn(acc[2], __uint_as_float(x0.z)); acc[3] = __fadd_rn(acc[3], __uint_as_float(x0.w));
-        acc[4] = __fadd_rn(acc[4], __uint_as_float(x1.x)); acc[5] = __fadd_rn(acc[5], __uint_as_float(x1.y));
-        acc[6] = __fadd_rn(acc[6], __uint_as_float(x1.z)); acc[7] = __fadd_rn(acc[7], __uint_as_float(x1.w));
+                                                unsigned int cnt, bool first, float (&acc)[16]) {
+  constexpr int G = BF16 ? 2 : 4;
+  constexpr unsigned int kRow = kRingTile * (BF16 ? 2u : 4u);
+  const unsigned int ng = cnt >> (BF16 ? 3 : 2);
+  bool act[G];
+#pragma unroll
+  for (int j = 0; j < G; ++j) act[j] = c + (unsigned int)j * kBulkConsumers < ng;
+#pragma unroll 2
+  for (unsigned int r = 0; r < nrows; ++r) {
+    const uint4* row = reinterpret_cast<const uint4*>(st + (size_t)r * kRow);
+    uint4 x[G];
+#pragma unroll
+    for (int j = 0; j < G; ++j) x[j] = act[j] ? row[c + (unsigned int)j * kBulkConsumers] : make_uint4(0, 0, 0, 0);
+    if (first && r == 0) {
+#pragma unroll
+      for (int j = 0; j < G; ++j) {
+        if (BF16) {
+          acc[8 * j + 0] = bf16_lo(x[j].x); acc[8 * j + 1] = bf16_hi(x[j].x);
+          acc[8 * j + 2] = bf16_lo(x[j].y); acc[8 * j + 3] = bf16_hi(x[j].y);
+          acc[8 * j + 4] = bf16_lo(x[j].z); acc[8 * j + 5] = bf16_hi(x[j].z);
+          acc[8 * j + 6] = bf16_lo(x[j].w); acc[8 * j + 7] = bf16_hi(x[j].w);
+        } else {
+          acc[4 * j + 0] = __uint_as_float(x[j].x); acc[4 * j + 1] = __uint_as_float(x[j].y);
+          acc[4 * j + 2] = __uint_as_float(x[j].z); acc[4 * j + 3] = __uint_as_float(x[j].w);
+        }
       }
-    }
-  } else {
-    const unsigned int ng = cnt >> 3;
-    const bool a0 = c < ng;
-    constexpr unsigned int kRow = kRingTile * 2;
-#pragma unroll 4
-    for (unsigned int r = 0; r < nrows; ++r) {
-      uint4 x = make_uint4(0, 0, 0, 0);
-      if (a0) x = reinterpret_cast<const uint4*>(st + (size_t)r * kRow)[c];
-      if (first && r == 0) {
-        widen8(x, acc);
-      } else {
-        add_bf16x2(acc[0], acc[1], x.x);
-        add_bf16x2(acc[2], acc[3], x.y);
-        add_bf16x2(acc[4], acc[5], x.z);
-        add_bf16x2(acc[6], acc[7], x.w);
+    } else {
+#pragma unroll
+      for (int j = 0; j < G; ++j) {
+        if (BF16) {
+          add_bf16x2(acc[8 * j + 0], acc[8 * j + 1], x[j].x);
+          add_bf16x2(acc[8 * j + 2], acc[8 * j + 3], x[j].y);
+          add_bf16x2(acc[8 * j + 4], acc[8 * j + 5], x[j].z);
+          add_bf16x2(acc[8 * j + 6], acc[8 * j + 7], x[j].w);
+        } else {
+          acc[4 * j + 0] = __fadd_rn(acc[4 * j + 0], __uint_as_float(x[j].x));
+          acc[4 * j + 1] = __fadd_rn(acc[4 * j + 1], __uint_as_float(x[j].y));
+          acc[4 * j + 2] = __fadd_rn(acc[4 * j + 2], __uint_as_float(x[j].z));
+          acc[4 * j + 3] = __fadd_rn(acc[4 * j + 3], __uint_as_float(x[j].w));
+        }
       }
     }
   }
@@ -160,20 +174,22 @@ __device__ __forceinline__ void ring_accumulate(unsigned int c, const unsigned c
 // The tile's last stage: parameters and state come out of the ring, the update goes to global memory.
 template <int OPT, bool BF16>
 __device__ __forceinline__ void ring_update(unsigned int c, const StageMeta& m, const unsigned char* __restrict__ st,
-                                            const float (&acc)[8], double& sq) {
+                                            const float (&acc)[16], double& sq) {
   const float4* rp = reinterpret_cast<const float4*>(st + m.state_off);
   const float4* ra = rp + kRingTile / 4;
   const float4* rb = ra + kRingTile / 4;
   const unsigned int ng4 = m.cnt >> 2;
   const float4 z = make_float4(0, 0, 0, 0);
-  // fp32: groups c and c + 256; bf16: groups 2c and 2c + 1 (the thread's 8 consecutive elements)
-  const unsigned int g0 = BF16 ? 2 * c : c, g1 = BF16 ? 2 * c + 1 : c + kBulkConsumers;
-  if (g0 < ng4)
-    update4<OPT>(m.h, make_float4(acc[0], acc[1], acc[2], acc[3]), m.p, m.s0, m.s1, (size_t)m.e0 + 4 * (size_t)g0,
-                 rp[g0], ra[g0], OPT == 1 ? rb[g0] : z, sq);
-  if (g1 < ng4)
-    update4<OPT>(m.h, make_float4(acc[4], acc[5], acc[6], acc[7]), m.p, m.s0, m.s1, (size_t)m.e0 + 4 * (size_t)g1,
-                 rp[g1], ra[g1], OPT == 1 ? rb[g1] : z, sq);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    // fp32: float4 group c + 256 q.  bf16: the thread's 16-byte group c + 256 (q / 2) holds the
+    // float4 groups 2 (c + 256 (q / 2)) and the next one.
+    const unsigned int g = BF16 ? 2u * (c + (unsigned int)(q >> 1) * kBulkConsumers) + (unsigned int)(q & 1)
+                                : c + (unsigned int)q * kBulkConsumers;
+    if (g < ng4)
+      update4<OPT>(m.h, make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]), m.p, m.s0, m.s1,
+                   (size_t)m.e0 + 4 * (size_t)g, rp[g], ra[g], OPT == 1 ? rb[g] : z, sq);
+  }
 }
 
 // ---- the kernel ----------------------------------------------------------------
@@ -187,8 +203,11 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
   __shared__ __align__(8) unsigned long long full_bar[kStages];
   __shared__ __align__(8) unsigned long long empty_bar[kStages];
   __shared__ __align__(16) StageMeta meta[kStages];
-  __shared__ double s_part[kStages][kBulkConsumerWarps];   // a chunk's sums of squares, one per consumer warp
-  __shared__ unsigned int s_pub_task[kStages], s_pub_chunk[kStages];
+  __shared__ __align__(8) unsigned long long pub_bar[kPubSlots];
+  __shared__ double s_part[kPubSlots][kBulkConsumerWarps];   // a chunk's sums of squares, one per consumer warp
+  __shared__ unsigned int s_pub_task[kPubSlots], s_pub_chunk[kPubSlots];
+  __shared__ unsigned int s_pub_done;      // chunks published so far (written by the publisher)
+  __shared__ unsigned int s_run_task[kPubRuns], s_run_chunks[kPubRuns];
   __shared__ int s_abort;
 
   PsTableHdr* hdr = reinterpret_cast<PsTableHdr*>(table);
@@ -204,6 +223,8 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
       mbar_init(&full_bar[s], 1);                       // the producer's arrive (+ transaction bytes)
       mbar_init(&empty_bar[s], kBulkConsumerWarps);     // one arrive per consumer warp
     }
+    for (int s = 0; s < kPubSlots; ++s) mbar_init(&pub_bar[s], kBulkConsumerWarps);
+    s_pub_done = 0;
     s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -214,45 +235,11 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
     // ------------------------------------------------------------ producer warp
     unsigned int cursor = 0, stage = 0, fills = 0;   // fills: stages posted so far
     unsigned int pend_mask = 0, pend_par = 0;        // stages whose last fill carried copies, and its parity
-    unsigned int pub_mask = 0, pub_par = 0;          // stages that closed a chunk whose partial sums are not published yet
+    unsigned int closed = 0;                         // chunks this CTA has closed (their last stage posted)
     bool ok = true;
     unsigned int idx = 0, next = 0;
     if (lane == 0) idx = atomicAdd(&hdr->counter, 1u);
     idx = __shfl_sync(0xffffffffu, idx, 0);
-
-    // Posts one stage: waits for the slot, publishes its description, arms the barrier and
-    // issues the copies (lane l fetches row l of the stage).  nsh shard rows from worker
-    // `first_w`, then nst state rows if this is the tile's last stage.
-    // The consumers leave a finished chunk's eight partial sums of squares in shared memory
-    // before they release the chunk's last stage; the producer publishes them when it next
-    // owns that stage.  (Published by the consumers themselves, the fence before the ticket
-    // made each of the eight warps wait for its own parameter stores once per chunk: the
-    // largest stall of the kernel.  The producer has no stores of its own in flight.)
-    auto publish = [&](unsigned int st) {
-      const unsigned int t = s_pub_task[st], c = s_pub_chunk[st];
-      const PsTaskDev* T = tasks + t;
-      const unsigned int first = T->first_chunk * kBulkConsumerWarps, n = T->nchunks * kBulkConsumerWarps;
-      if (lane < kBulkConsumerWarps) __stcg(partials + (size_t)c * kBulkConsumerWarps + lane, s_part[st][lane]);
-      __syncwarp();
-      unsigned int done = 0;
-      if (lane == 0) {
-        __threadfence();
-        done = atomicAdd(&tasks[t].ticket, (unsigned int)kBulkConsumerWarps);
-        __threadfence();
-      }
-      done = __shfl_sync(0xffffffffu, done, 0);
-      if (done == n - kBulkConsumerWarps) {
-        const double tot = sum_partials_warp(partials + first, n, lane);
-        if (lane == 0) {
-          PsStat stt;
-          stt.sqnorm = tot;
-          stt.step = T->step;
-          stt.busy_ns = 0; stt.t_first = 0; stt.t_last = 0; stt._r0 = 0;
-          stats[T->stat_idx] = stt;
-        }
-      }
-      pub_mask &= ~(1u << st);
-    };
 
     // what every stage of a chunk repeats, read from the table once per chunk
     struct ChunkCtx {
@@ -263,13 +250,31 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
       unsigned int ges, nstate_rows;
     } cc = {};
 
+    // A finished chunk's partial sums go to slot closed % kPubSlots: free once the publisher is
+    // fewer than kPubSlots chunks behind (it normally is: a publish costs a few microseconds,
+    // a chunk several).
+    auto slot_free = [&]() {
+      const volatile unsigned int* pd = &s_pub_done;
+      if (closed - *pd >= (unsigned int)kPubSlots) {
+        const long long t0 = clock64();
+        while (closed - *pd >= (unsigned int)kPubSlots) {
+          if (*const_cast<volatile int*>(&s_abort) || clock64() - t0 > wait_limit) { ok = false; break; }
+        }
+      }
+      ok = __all_sync(0xffffffffu, ok);
+      return ok;
+    };
+
+    // Posts one stage: waits for the slot, writes its description, arms the barrier and
+    // issues the copies (lane l fetches row l of the stage): nsh shard rows from worker
+    // `first_w`, then the state rows if this is the tile's last stage.
     auto post = [&](unsigned int task, unsigned int chunk, size_t e0,
                     unsigned int cnt, unsigned int first_w, unsigned int nsh, bool with_state, unsigned int flags) {
       const unsigned int use = fills / kStages;
       if (use > 0) ok = mbar_wait(&empty_bar[stage], (use - 1) & 1u, &s_abort, wait_limit);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) return;
-      if ((pub_mask >> stage) & 1u) publish(stage);
+      if ((flags & kChunkEnd) && !slot_free()) return;
       const unsigned int ges = cc.ges;
       const unsigned int nst = with_state ? cc.nstate_rows : 0u;
       const unsigned int row_slot = kRingTile * ges;
@@ -282,20 +287,18 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
         m.task = task; m.chunk = chunk; m.cnt = cnt; m.nrows = nsh;
         m.state_off = nsh * row_slot;
         m.flags = flags;
+        m.pub_slot = closed % (unsigned int)kPubSlots;
         m.W = cc.W;
         m.kind = cc.kind;
         m.h = cc.h;
         if (flags & kChunkEnd) {
-          s_pub_task[stage] = task;
-          s_pub_chunk[stage] = chunk;
+          s_pub_task[m.pub_slot] = task;
+          s_pub_chunk[m.pub_slot] = chunk;
         }
         if (bytes) mbar_arrive_expect_tx(&full_bar[stage], bytes);
         else mbar_arrive(&full_bar[stage]);
       }
-      if (flags & kChunkEnd) {
-        pub_mask |= 1u << stage;
-        pub_par = (pub_par & ~(1u << stage)) | ((use & 1u) << stage);
-      }
+      if (flags & kChunkEnd) ++closed;
       __syncwarp();
       if (bytes) {
         if (lane < nsh) {
@@ -356,23 +359,21 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
       }
       idx = __shfl_sync(0xffffffffu, next, 0);
     }
-    // end marker for the consumers
+    // end marker for the consumers; the publisher learns how many chunks to expect
     if (ok) {
       const unsigned int use = fills / kStages;
       if (use > 0) ok = mbar_wait(&empty_bar[stage], (use - 1) & 1u, &s_abort, wait_limit);
       ok = __all_sync(0xffffffffu, ok);
-      if (ok) {
-        if ((pub_mask >> stage) & 1u) publish(stage);
-        if (lane == 0) {
-          meta[stage].flags = kTileEnd;
-          mbar_arrive(&full_bar[stage]);
-        }
-        // the chunks that ended in the other stages: published once the consumers have released them
-        for (unsigned int st = 0; ok && st < (unsigned int)kStages; ++st) {
-          if (!((pub_mask >> st) & 1u)) continue;
-          ok = __all_sync(0xffffffffu, mbar_wait(&empty_bar[st], (pub_par >> st) & 1u, &s_abort, wait_limit));
-          if (ok) publish(st);
-        }
+      if (ok && lane == 0) {
+        meta[stage].flags = kTileEnd;
+        mbar_arrive(&full_bar[stage]);
+      }
+      // and for the publisher: a slot whose task is the end mark, armed in the consumers' stead
+      if (ok && slot_free()) {
+        const unsigned int slot = closed % (unsigned int)kPubSlots;
+        if (lane == 0) s_pub_task[slot] = kPubEnd;
+        __syncwarp();
+        if (lane < kBulkConsumerWarps) mbar_arrive(&pub_bar[slot]);
       }
     }
     if (!ok && lane == 0) {
@@ -387,13 +388,100 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
         }
     }
     __syncwarp();
+  } else if (warp == kBulkConsumerWarps + 1) {
+    // ------------------------------------------------------------ publisher warp
+    // Chunk k of this CTA leaves its eight partial sums in slot k % kPubSlots; each consumer
+    // warp arrives on the slot's barrier once its share is there.  This warp copies them to
+    // global memory and remembers which task they belong to.  The tickets that count a
+    // task's chunks — and with them the fences — are drawn once per kPubRuns chunks (and
+    // when the CTA runs out of work): a memory fence executed by ANY warp of the SM while
+    // bulk copies are in flight slows the ring down (10 % of its throughput with two
+    // fences per chunk, measured with the fences here, in the producer, and left out).
+    // Whoever draws a task's last ticket adds its partial sums up in a fixed order; doing
+    // all of that at the CTA's end instead would leave the sums of most tasks to the few
+    // CTAs that finish last (tried: 30 % slower).
+    unsigned int nruns = 0, run_task = kPubEnd, since = 0;
+    auto write_stat = [&](const PsTaskDev* T, double tot) {
+      PsStat stt;
+      stt.sqnorm = tot;
+      stt.step = T->step;
+      stt.busy_ns = 0; stt.t_first = 0; stt.t_last = 0; stt._r0 = 0;
+      stats[T->stat_idx] = stt;
+    };
+    auto flush = [&]() {
+      __syncwarp();
+      if (nruns == 0) return;
+      __threadfence();                                  // this warp's partial sums before its tickets
+      const unsigned int i = lane;                      // (kPubRuns <= 32: one lane per run)
+      const bool have = i < nruns;
+      const unsigned int t = have ? s_run_task[i] : 0u;
+      const unsigned int add = have ? s_run_chunks[i] : 0u;
+      bool last = false;
+      if (have) last = atomicAdd(&tasks[t].ticket, add) + add == tasks[t].nchunks;
+      unsigned int todo = __ballot_sync(0xffffffffu, last);
+      if (todo) __threadfence();                        // the other CTAs' partial sums after the ticket
+      while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const PsTaskDev* T = tasks + __shfl_sync(0xffffffffu, t, src);
+        const double tot = sum_partials_warp(partials + T->first_chunk, T->nchunks, lane);
+        if (lane == 0) write_stat(T, tot);
+      }
+      nruns = 0;
+      run_task = kPubEnd;
+      __syncwarp();
+    };
+    for (unsigned int k = 0;; ++k) {
+      const unsigned int slot = k % (unsigned int)kPubSlots, parity = (k / (unsigned int)kPubSlots) & 1u;
+      if (!__all_sync(0xffffffffu, mbar_wait(&pub_bar[slot], parity, &s_abort, wait_limit))) {
+        if (lane == 0) {
+          s_abort = 1;
+          atomicExch(status, 3);
+        }
+        break;
+      }
+      const unsigned int t = s_pub_task[slot], c = s_pub_chunk[slot];
+      if (t == kPubEnd) {
+        flush();
+        break;
+      }
+      // the chunk's sum of squares: its eight shares added in warp order
+      double sum = 0.0;
+      if (lane == 0) {
+#pragma unroll
+        for (int w = 0; w < kBulkConsumerWarps; ++w) sum += s_part[slot][w];
+      }
+      const PsTaskDev* T = tasks + t;
+      if (T->nchunks == 1) {                            // nobody else to wait for: no ticket, no fence
+        if (lane == 0) write_stat(T, sum);
+      } else {
+        if (lane == 0) __stcg(partials + c, sum);
+        if (since == (unsigned int)kPubRuns) {
+          flush();
+          since = 0;
+        }
+        ++since;
+        if (t != run_task) {                            // consecutive chunks of one task share a ticket draw
+          if (lane == 0) {
+            s_run_task[nruns] = t;
+            s_run_chunks[nruns] = 0;
+          }
+          run_task = t;
+          ++nruns;
+        }
+        __syncwarp();
+        if (lane == 0) ++s_run_chunks[nruns - 1];
+      }
+      __syncwarp();
+      if (lane == 0) *const_cast<volatile unsigned int*>(&s_pub_done) = k + 1;    // the slot may be filled again
+    }
   } else {
     // -------------------------------------------------------------- consumer warps
     unsigned int stage = 0, takes = 0;
     double sq = 0.0;
-    float acc[8];
+    float acc[16];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+    for (int k = 0; k < 16; ++k) acc[k] = 0.f;
     while (true) {
       // all lanes poll; the outcome is made warp-uniform before anyone leaves
       if (!__all_sync(0xffffffffu, mbar_wait(&full_bar[stage], (takes / kStages) & 1u, &s_abort, wait_limit))) {
@@ -446,10 +534,13 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
         }
       }
       if (flags & kChunkEnd) {
-        // this warp's share of the chunk's sum of squares, left for the producer to publish
+        // this warp's share of the chunk's sum of squares, left for the publisher warp
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) sq += __shfl_down_sync(0xffffffffu, sq, o);
-        if (lane == 0) s_part[stage][warp] = sq;
+        if (lane == 0) {
+          s_part[m.pub_slot][warp] = sq;
+          mbar_arrive(&pub_bar[m.pub_slot]);
+        }
         sq = 0.0;
       }
       __syncwarp();
