@@ -41,6 +41,7 @@ constexpr int kStageBytes = 49152;
 constexpr int kStages = 4;
 constexpr int kBulkSmemBytes = kStages * kStageBytes + 1024;
 constexpr unsigned int kRingTile = 4096;                    // elements per tile: 16 per consumer thread
+static_assert(3u * kRingTile * 4u <= (unsigned int)kStageBytes, "a stage holds p and two state rows of a tile");
 constexpr long long kDrainCycles = 4000000000ll;            // limit of the producer's own wait for its copies (about 2 s)
 constexpr unsigned int kWaitUnit = 1024;                    // the table gives its wait limit in units of this many cycles
 
