@@ -292,12 +292,14 @@ class FullPair:
     bench.py times (overlapped launches, rounds given with their inputs
     complete, packing over time)."""
 
-    def __init__(self, cfg: configs.Config, device: int = 0, overlap: int = 1):
+    def __init__(self, cfg: configs.Config, device: int = 0, overlap: int = 1, kernel: int = 0):
         self.cfg = cfg
         self.dev = torch.device("cuda", device)
         arena = sum(3 * (4 * b.nelem + 256) for j in cfg.jobs for b in j.blocks) + (64 << 20)
         self.svc = B.Service(device, cfg.num_contexts, arena)
         self.svc.set_option(B.PS_OPT_OVERLAP, overlap)
+        if kernel:
+            self.svc.set_option(B.PS_OPT_KERNEL, kernel)
         self.ora = A.OracleAggregator(cfg.num_contexts, 0)
         self.ctx = {}
         for j, job in enumerate(cfg.jobs):

@@ -74,6 +74,25 @@ def test_c3_vgg16_shaped_20_iterations_every_element():
         pair.close()
 
 
+@pytest.mark.parametrize("name", ["C3", "C5"])
+def test_ring_kernel_on_full_size_shapes_every_element(name):
+    """The bulk-copy ring kernel (PS_OPT_KERNEL = 2) on the VGG-16-shaped job (fp32, SGD, W = 16)
+    and the BERT-large-shaped one (bf16, Adam, W = 32, two contexts): three iterations, every
+    element and every block's norm compared after the first and the last — full-size launches
+    are where a CTA closes hundreds of chunks and its publisher warp draws tickets in batches."""
+    cfg = configs.CONFIGS[name]()
+    pair = FullPair(cfg, kernel=2)
+    try:
+        rounds = configs.rounds_all(cfg)
+        for it in range(3):
+            pair.iteration(it, rounds)
+            if it in (0, 2):
+                assert pair.compare(it + 1) == cfg.num_params
+        assert pair.svc.launch_info()["kernel"] == "bulk"
+    finally:
+        pair.close()
+
+
 @pytest.mark.parametrize("overlap", [0, 1], ids=["in-stream", "overlapped"])
 def test_c4_twelve_packed_jobs_bursty_arrival_every_element(overlap):
     cfg = configs.c4()
