@@ -319,28 +319,70 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
       stage = (stage + 1 == kStages) ? 0 : stage + 1;
     };
 
+    // What the producer reads from a task's record.  The record of the NEXT chunk's task is
+    // requested while the current chunk streams (its claim is issued at the top of the chunk):
+    // found and read only when the chunk starts, the table look-ups — a chain of three or four
+    // dependent trips to L2 — kept the producer busy for a third of a W = 4 chunk.
+    struct TaskRegs {
+      float *p, *s0, *s1;
+      unsigned long long nelem;
+      unsigned int shard_row, first_chunk, vec_ok, tile_elems, chunk_elems;
+      int job;
+      float ss_t, sbc2_t;
+    };
+    auto load_task = [&](unsigned int t) {
+      const PsTaskDev* T = tasks + t;
+      TaskRegs r;
+      r.p = T->p; r.s0 = T->s0; r.s1 = T->s1;
+      r.nelem = T->nelem;
+      r.shard_row = T->shard_row; r.first_chunk = T->first_chunk;
+      r.vec_ok = T->vec_ok; r.tile_elems = T->tile_elems; r.chunk_elems = T->chunk_elems;
+      r.job = T->job;
+      r.ss_t = T->ss_t; r.sbc2_t = T->sbc2_t;
+      return r;
+    };
+    TaskRegs tr = {}, ntr = {};
+    unsigned int ncursor = 0;
+    bool looked = true;
+    auto look_ahead = [&]() {            // once per chunk, after its first stages are on their way
+      if (looked) return;
+      looked = true;
+      next = __shfl_sync(0xffffffffu, next, 0);
+      ncursor = cursor;
+      ntr = tr;
+      if (next < total) {
+        ncursor = find_task(starts, n_tasks, cursor, next, lane);
+        if (ncursor != cursor) ntr = load_task(ncursor);
+      }
+    };
+    if (idx < total) {
+      cursor = find_task(starts, n_tasks, cursor, idx, lane);
+      tr = load_task(cursor);
+    }
+
     while (ok && idx < total) {
       if (lane == 0) next = atomicAdd(&hdr->counter, 1u);      // overlaps this chunk's copies
-      cursor = find_task(starts, n_tasks, cursor, idx, lane);
-      const PsTaskDev* T = tasks + cursor;
-      const PsJobDev* J = jobs + T->job;
+      looked = false;
+      const PsJobDev* J = jobs + tr.job;
       const unsigned int W = (unsigned int)J->W;
       const unsigned int ges = J->grad_dtype ? 2u : 4u;
       const unsigned int vecw = J->grad_dtype ? 8u : 4u;
       const unsigned int state_bytes = (J->opt ? 3u : 2u) * kRingTile * 4u;
       const unsigned int rows_per_stage = kStageBytes / (kRingTile * ges);
-      const unsigned int chunk_elems = T->chunk_elems;
-      const size_t begin = (size_t)(idx - T->first_chunk) * chunk_elems;
-      const unsigned int count = (unsigned int)min((unsigned long long)chunk_elems, T->nelem - begin);
+      const unsigned int chunk_elems = tr.chunk_elems;
+      const size_t begin = (size_t)(idx - tr.first_chunk) * chunk_elems;
+      const unsigned int count = (unsigned int)min((unsigned long long)chunk_elems, tr.nelem - begin);
       const unsigned int body = count & ~(vecw - 1);
-      cc.h = load_hp(J, T);
-      cc.p = T->p; cc.s0 = T->s0; cc.s1 = T->s1;
-      cc.shards = ptrs + T->shard_row;
+      cc.h.lr = J->lr; cc.h.mom = J->mom; cc.h.wd = J->wd; cc.h.b1 = J->b1; cc.h.b2 = J->b2;
+      cc.h.omb1 = J->omb1; cc.h.omb2 = J->omb2; cc.h.eps = J->eps; cc.h.gs = J->gs;
+      cc.h.ss_t = tr.ss_t; cc.h.sbc2_t = tr.sbc2_t;
+      cc.p = tr.p; cc.s0 = tr.s0; cc.s1 = tr.s1;
+      cc.shards = ptrs + tr.shard_row;
       cc.W = J->W;
       cc.kind = (J->opt << 1) | J->grad_dtype;
       cc.ges = ges;
       cc.nstate_rows = J->opt ? 3u : 2u;
-      if (T->tile_elems == 0 || T->vec_ok == 0 || body == 0) {
+      if (tr.tile_elems == 0 || tr.vec_ok == 0 || body == 0) {
         post(cursor, idx, begin, 0u, 0u, 0u, false, kTileDirect | kChunkEnd);
       } else {
         for (unsigned int off = 0; ok && off < body; off += kRingTile) {
@@ -355,10 +397,14 @@ ps_aggregate_bulk_kernel(unsigned char* __restrict__ table, const PsJobDev* __re
             w += nsh;
             if (ok && last_rows && !with_state)       // the state rows get a stage of their own
               post(cursor, idx, begin + off, cnt, W, 0u, true, kTileLast | end_flag);
+            look_ahead();
           }
         }
       }
-      idx = __shfl_sync(0xffffffffu, next, 0);
+      look_ahead();
+      idx = next;
+      cursor = ncursor;
+      tr = ntr;
     }
     // end marker for the consumers; the publisher learns how many chunks to expect
     if (ok) {

@@ -496,7 +496,7 @@ int build_plan(ps_service* s, const std::vector<int>& idx, Plan* plan) {
   h->tasks_off = (unsigned int)tasks_off;
   h->starts_off = (unsigned int)starts_off;
   h->ptrs_off = (unsigned int)ptrs_off;
-  h->parts_per_chunk = (use_bulk(s) && !plan->has_sparse) ? kBulkConsumerWarps : 1;
+  h->parts_per_chunk = 1;
   h->profile = s->opt_profile ? 1u : 0u;
   h->sparse_off = (unsigned int)sparse_off;
   h->exited = 0;
@@ -1076,7 +1076,7 @@ static int launch_plan(ps_service* s, const std::vector<int>& idx, Plan& plan, c
   const bool inl = s->opt_inline && !bulk && !plan.has_sparse && plan.bytes.size() <= kInlineBytes &&
                    plan.total_chunks <= (unsigned int)(kInlineGridFactor * grid_cap(s));
   rc = acquire_slot(s, inl ? 0 : plan.bytes.size(),
-                    (size_t)plan.total_chunks * (bulk ? kBulkConsumerWarps : 1), &sl);
+                    (size_t)plan.total_chunks, &sl);
   if (rc) return rc;
   const int slot_index = (int)(sl - s->slots);
   // Overlap mode: the launch goes to one of the service-owned streams, after the
