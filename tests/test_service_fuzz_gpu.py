@@ -31,6 +31,8 @@ def test_random_operation_sequences(seed):
     nctx = 3
     svc = B.Service(0, nctx, 64 << 20)
     svc.set_option(B.PS_OPT_OVERLAP, seed % 2)          # odd seeds: launches on the service's own streams
+    if (seed >> 1) & 1:                                 # seeds 2, 3, 6, 7, ...: the bulk-copy ring kernel
+        svc.set_option(B.PS_OPT_KERNEL, 2)
     ora = A.OracleAggregator(nctx)
     streams = [None, torch.cuda.Stream(), torch.cuda.Stream()]
     jobs, blocks = [], {}            # blocks[(j, b)] = dict(n, rows, pushed=set)
