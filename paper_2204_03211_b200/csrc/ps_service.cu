@@ -356,6 +356,13 @@ int grid_cap(ps_service* s) {
   return s->num_sms * per_sm;
 }
 
+// One "wave" of work for the packing and splitting rules, in chunks: what the direct-load
+// kernel's resident CTAs take at once.  A CTA of the ring kernel has an SM to itself and
+// streams as much as four of those, so its waves are counted in the same unit.
+unsigned long long work_wave(ps_service* s) {
+  return use_bulk(s) ? 4ull * (unsigned long long)s->num_sms : (unsigned long long)grid_cap(s);
+}
+
 // Automatic chunk size.  Measured on B200 (C2, C4 all-ready and C4 in bursty
 // rounds): 8192 elements beats 2048/4096/16384 and beats shrinking the chunks
 // toward the end of the table; the per-launch cost that remains (about 30 us)
@@ -1210,7 +1217,7 @@ int parts_for(ps_service* s, const std::vector<int>& idx) {
   if (!s->opt_overlap || !s->opt_split) return 1;
   unsigned long long chunks = 0;
   for (int bi : idx) chunks += (s->blocks[bi].nelem + kChunkAuto - 1) / kChunkAuto;
-  const unsigned long long per = kSplitWavesX2 * (unsigned long long)grid_cap(s) / 2;
+  const unsigned long long per = kSplitWavesX2 * work_wave(s) / 2;
   return (int)std::max<unsigned long long>(1, std::min<unsigned long long>(kSplitMax, chunks / per));
 }
 
@@ -1313,7 +1320,7 @@ static int submit_ready(ps_service* s, const std::vector<int>& idx, cudaStream_t
   // (12 packed jobs, bursty: 4.62 ms per step); holding back until the device runs dry
   // turns a step of 54 small rounds into one launch with no tail to overlap (0.21 ms);
   // this rule gives 4.44 ms and 0.18 ms.
-  const unsigned long long wave = (unsigned long long)grid_cap(s);
+  const unsigned long long wave = work_wave(s);
   if (!busy || (s->batch_chunks >= kBatchSend * wave && unfinished_launches(s) < kBatchAhead) ||
       s->batch_chunks >= kBatchMust * wave)
     return flush_batch(s);
