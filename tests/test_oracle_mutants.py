@@ -1,0 +1,125 @@
+"""Do the oracle's pins have teeth?  Plausible mistakes are planted in a COPY
+of the oracle's source, one at a time (a wrong sign, a swapped operand, a
+dropped worker or term, eps inside the root, a missing bias correction, a
+wrong half of the bf16 word, ...), the copy is compiled, and the pin files
+are run against it in a child process: every one of them has to fail.  Each
+mistake is planted in the binary32 AND the binary64 mode, so that the pin
+"binary32 tracks binary64" cannot be what catches it: a closed form, a
+hand-worked value or an invariant has to.
+
+The mistakes live on the CPU, in the checker; nothing here touches the GPU.
+"""
+import os
+import subprocess
+import sys
+from concurrent.futures import ThreadPoolExecutor
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = os.path.join(ROOT, "oracle", "ps_oracle.cpp")
+PINS = ["tests/test_oracle_pins.py", "tests/test_oracle_ieee.py"]
+
+# name -> [(text in the oracle's source, replacement), ...]; every text must occur
+MUTANTS = {
+    "reduce: a worker subtracted": [
+        ("G = G + shard_value(hp, k->shards[w], i);", "G = G - shard_value(hp, k->shards[w], i);"),
+        ("G = G + (double)shard_value(hp, k->shards[w], i);", "G = G - (double)shard_value(hp, k->shards[w], i);")],
+    "reduce: last worker dropped": [("for (int w = 1; w < W; ++w)", "for (int w = 1; w + 1 < W; ++w)")],
+    "reduce: worker index off by one": [("k->shards[w], i)", "k->shards[w - 1], i)")],
+    "reduce: mean instead of sum": [("G = G * gs;", "G = G * gs / W;")],
+    "grad_scale dropped": [("G = G * gs;", "G = G * 1;")],
+    "decay applied to the state": [("wd * p[i]", "wd * s0[i]")],
+    "decay subtracted": [("const float d = G + wdp;", "const float d = G - wdp;"),
+                         ("const double d = G + wd * p[i];", "const double d = G - wd * p[i];")],
+    "decay dropped": [("const float d = G + wdp;", "const float d = G;"),
+                      ("const double d = G + wd * p[i];", "const double d = G;")],
+    "momentum taken from the parameter": [("mom * s0[i]", "mom * p[i]")],
+    "velocity: gradient subtracted": [("const float v = mv + d;", "const float v = mv - d;"),
+                                      ("const double v = mom * s0[i] + d;", "const double v = mom * s0[i] - d;")],
+    "sgd: step from the gradient, not the velocity": [("const float step = lr * v;", "const float step = lr * d;"),
+                                                       ("p[i] = p[i] - lr * v;", "p[i] = p[i] - lr * d;")],
+    "sgd: lr inside the velocity": [("const float v = mv + d;", "const float v = mv + lr * d;"),
+                                    ("const float step = lr * v;", "const float step = v;"),
+                                    ("const double v = mom * s0[i] + d;", "const double v = mom * s0[i] + lr * d;"),
+                                    ("p[i] = p[i] - lr * v;", "p[i] = p[i] - v;")],
+    "ascent instead of descent": [("p[i] = p[i] - step;", "p[i] = p[i] + step;"),
+                                  ("p[i] = p[i] - lr * v;", "p[i] = p[i] + lr * v;"),
+                                  ("p[i] = p[i] - ss_t * (m / den);", "p[i] = p[i] + ss_t * (m / den);")],
+    "sgd: velocity not stored": [("      s0[i] = v;\n", "      ;\n")],
+    "adam: beta2 on the first moment": [("b1 * s0[i]", "b2 * s0[i]")],
+    "adam: beta1 instead of 1 - beta1": [("omb1 * d", "b1 * d")],
+    "adam: gradient not squared": [("const float dd = d * d;", "const float dd = d;"),
+                                   ("omb2 * (d * d)", "omb2 * (d)")],
+    "adam: beta1 on the second moment": [("b2 * s1[i]", "b1 * s1[i]")],
+    "adam: beta2 instead of 1 - beta2": [("const float odd = omb2 * dd;", "const float odd = b2 * dd;"),
+                                         ("omb2 * (d * d)", "b2 * (d * d)")],
+    "adam: no square root": [("std::sqrt(v)", "(v)")],
+    "adam: second bias correction multiplied": [("const float rh = r / sbc2_t;", "const float rh = r * sbc2_t;"),
+                                                ("std::sqrt(v) / sbc2_t", "std::sqrt(v) * sbc2_t")],
+    "adam: second bias correction dropped": [("const float rh = r / sbc2_t;", "const float rh = r;"),
+                                             ("std::sqrt(v) / sbc2_t", "std::sqrt(v)")],
+    "adam: eps dropped": [("const float den = rh + eps;", "const float den = rh;"),
+                          ("/ sbc2_t + eps;", "/ sbc2_t;")],
+    "adam: eps inside the root": [("const float r = std::sqrt(v);", "const float r = std::sqrt(v + eps);"),
+                                  ("const float den = rh + eps;", "const float den = rh;"),
+                                  ("const double den = std::sqrt(v) / sbc2_t + eps;",
+                                   "const double den = std::sqrt(v + eps) / sbc2_t;")],
+    "adam: quotient inverted": [("m / den", "den / m")],
+    "adam: first bias correction dropped": [("(float)oracle_adam_step_size(lr, b1, k->step)", "lr"),
+                                            ("= oracle_adam_step_size(hp->lr, hp->beta1, k->step)", "= lr")],
+    "adam: first bias correction with the wrong sign": [
+        ("(double)lr / (1.0 - std::pow((double)beta1, (double)t))", "(double)lr / (1.0 + std::pow((double)beta1, (double)t))")],
+    "adam: first bias correction with beta^(t-1)": [
+        ("(double)lr / (1.0 - std::pow((double)beta1, (double)t))", "(double)lr / (1.0 - std::pow((double)beta1, (double)t + 1.0))")],
+    "adam: second bias correction without its root": [
+        ("return std::sqrt(1.0 - std::pow((double)beta2, (double)t));", "return 1.0 - std::pow((double)beta2, (double)t);")],
+    "adam: first moment not stored": [("      s0[i] = m;\n", "      ;\n")],
+    "adam: second moment not stored": [("      s1[i] = v;\n", "      ;\n")],
+    "adam: decay decoupled from the moments": [
+        ("      const float q = m / den;\n      const float step = ss_t * q;",
+         "      const float q = m / den;\n      const float step = ss_t * q + lr * wdp;"),
+        ("const float od = omb1 * d;", "const float od = omb1 * G;"),
+        ("const float dd = d * d;", "const float dd = G * G;"),
+        ("const double m = b1 * s0[i] + omb1 * d;", "const double m = b1 * s0[i] + omb1 * G;"),
+        ("const double v = b2 * s1[i] + omb2 * (d * d);", "const double v = b2 * s1[i] + omb2 * (G * G);"),
+        ("p[i] = p[i] - ss_t * (m / den);", "p[i] = p[i] - ss_t * (m / den) - lr * wd * p[i];")],
+    "norm: not squared": [("sq += (double)G * (double)G;", "sq += (double)G;"), ("sq += G * G;", "sq += G;")],
+    "norm: taken before the scale": [("    G = G * gs;\n    sq += (double)G * (double)G;", "    sq += (double)G * (double)G;\n    G = G * gs;"),
+                                     ("    G = G * gs;\n    sq += G * G;", "    sq += G * G;\n    G = G * gs;")],
+    "bf16: shifted by 15": [("(uint32_t)bits << 16", "(uint32_t)bits << 15")],
+    "bf16: low half of the word": [("(uint32_t)bits << 16", "(uint32_t)bits")],
+}
+
+
+def _build(tmp, name, edits):
+    src = open(SRC).read()
+    for old, new in edits:
+        assert src.count(old) >= 1, "mutant %r: text %r not in the oracle's source" % (name, old)
+        src = src.replace(old, new)
+    stem = "".join(c if c.isalnum() else "_" for c in name)
+    cpp, lib = os.path.join(tmp, stem + ".cpp"), os.path.join(tmp, "lib" + stem + ".so")
+    open(cpp, "w").write(src)
+    subprocess.run(["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-fPIC", "-shared",
+                    "-w", "-o", lib, cpp], check=True)
+    return lib
+
+
+def _pins_pass(lib):
+    """Runs the pin files in a child whose oracle loads `lib`; True if they all pass."""
+    code = ("import sys; sys.path.insert(0, %r); import oracle.build as ob; ob.build = lambda force=False: %r; "
+            "import pytest; sys.exit(pytest.main(['-x', '-q', '-p', 'no:cacheprovider'] + %r))" % (ROOT, lib, PINS))
+    r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, capture_output=True, text=True,
+                       env=dict(os.environ, OMP_NUM_THREADS="2"))
+    assert r.returncode in (0, 1), "the pin run itself broke:\n" + r.stdout[-2000:] + r.stderr[-2000:]
+    return r.returncode == 0
+
+
+def test_every_planted_mistake_fails_a_pin(tmp_path):
+    tmp = str(tmp_path)
+    assert _pins_pass(_build(tmp, "control", [])), "the unchanged oracle must pass its pins"
+    names = list(MUTANTS)
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        survived = [n for n, ok in zip(names, pool.map(lambda n: _pins_pass(_build(tmp, n, MUTANTS[n])), names)) if ok]
+    assert not survived, "no pin notices: " + "; ".join(survived)
+    assert len(names) >= 30
