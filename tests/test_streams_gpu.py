@@ -64,9 +64,11 @@ def test_migration_without_room_fails_cleanly_and_block_keeps_working():
 
 
 @pytest.mark.parametrize("dt", [configs.F32, configs.BF16])
-def test_maximum_worker_count(dt):
+@pytest.mark.parametrize("kernel", [1, 2, 3], ids=["ldg", "bulk", "inline"])
+def test_maximum_worker_count(dt, kernel):
+    # (the ring kernel takes W = 256 in 86 fp32 or 43 bf16 stages per tile)
     cfg = tiny_config([4096 + 3, 9000], B.PS_MAX_WORKERS, grad_dtype=dt, grad_std=1e-3)
-    pair = Pair(cfg)
+    pair = Pair(cfg, kernel=kernel)
     try:
         for it in range(2):
             pair.push_iteration(it)
