@@ -118,7 +118,7 @@ def test_two_gloo_ranks_agree_on_owners_and_split_the_registry(tmp_path):
         assert abs(got["elems"][0] - got["elems"][1]) <= 0.02 * cfg.num_params
 
 
-def _gpu_rank(rank, world, port, out, transport="inplace"):
+def _gpu_rank(rank, world, port, out, transport="inplace", kernel=0):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
     dist.init_process_group("gloo", rank=rank, world_size=world)
     from helpers import oracle_hp, tiny_config, to_np
@@ -136,6 +136,8 @@ def _gpu_rank(rank, world, port, out, transport="inplace"):
     cfg = configs.Config("sharded-tiny", 321, 3, [a, b])
     wl = bench_sharded.ShardedWorkload(cfg, rank, world, 0, exchange, dist.barrier, arena_slack=16 << 20,   # room for adopted blocks
                                        transport=transport)
+    if kernel:
+        wl.sh.svc.set_option(B.PS_OPT_KERNEL, kernel)
     # the oracle of each rank follows EVERY block (they are tiny), so that a block
     # adopted by this rank half-way has its history
     ora = A.OracleAggregator(1, 0)
@@ -244,6 +246,18 @@ def test_two_processes_on_one_device_read_each_others_shards_in_place(tmp_path):
     assert all(g["checked"] + g["pulled"] == 9 for g in got)       # the rest was pulled from the other rank's arena
     assert all(g["remote_reads"] > 0 for g in got)                 # each rank consumed shards hosted by the other
     assert all(g["adopted"] >= 2 and g["sent"] > 0 for g in got)   # and blocks changed owner in both directions
+
+
+@pytest.mark.gpu
+def test_two_processes_on_one_device_ring_kernel_reads_mapped_shards(tmp_path):
+    """In place again, with the bulk-copy ring kernel: its copies into shared memory
+    start at addresses mapped from the other process's buffer (no multicast anywhere)."""
+    out = str(tmp_path / "r%d.json")
+    mp.spawn(_gpu_rank, args=(2, _free_port(), out, "inplace", 2), nprocs=2, join=True)
+    got = [json.load(open(out % r)) for r in range(2)]
+    assert all(g["ok"] and g["status"] == 0 for g in got), got
+    assert sum(g["checked"] for g in got) == 9 and all(g["remote_reads"] > 0 for g in got)
+    assert all(g["adopted"] >= 2 and g["sent"] > 0 for g in got)
 
 
 @pytest.mark.gpu
