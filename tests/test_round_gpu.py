@@ -339,3 +339,65 @@ def test_rounds_held_back_behind_a_busy_device_are_packed_and_lose_nothing(prepa
         pair.compare()
     finally:
         pair.close()
+
+
+def test_four_host_threads_each_drive_a_job_through_the_same_service():
+    """Many jobs' Agents talk to one Aggregator at once (paper, Section 3.1): four host
+    threads, one per job, each with its own stream, send their job's rounds (three
+    blocks at a time, inputs complete) for three iterations with no coordination
+    between them; calls are serialised inside the service, rounds of different jobs
+    interleave and pack as they come.  Every element of every block must come out as
+    the oracle's, whatever the interleaving was."""
+    import threading
+    from helpers import FullPair
+    jobs = [tiny_config([70001, 5, 4096, 300000, 33, 1 << 20, 12289], 3).jobs[0],
+            tiny_config([1 << 18, 12289, 1, 8192, 555555], 4, opt=configs.ADAM, grad_dtype=configs.BF16).jobs[0],
+            tiny_config([2_000_003, 64, 4099], 8, momentum=0.0).jobs[0],
+            tiny_config([100000] * 9, 2, opt=configs.ADAM, weight_decay=1e-2).jobs[0]]
+    cfg = configs.Config("threads", 77, 3, jobs)
+    pair = FullPair(cfg)
+    svc = pair.svc
+    iters = 3
+    try:
+        slabs = [[generate.grad_slab(cfg, j, it, pair.dev) for it in range(iters)] for j in range(len(jobs))]
+        torch.cuda.synchronize()
+        errors, start = [], threading.Barrier(len(jobs))
+
+        def agent(j):
+            try:
+                job, stream = cfg.jobs[j], torch.cuda.Stream()
+                start.wait()
+                for it in range(iters):
+                    blocks = [b.block for b in job.blocks]
+                    for k in range(0, len(blocks), 3):
+                        ready = [(j, b) for b in blocks[k:k + 3]]
+                        js, bs, ws, ps = [], [], [], []
+                        for (_, b) in ready:
+                            for w in range(job.num_workers):
+                                js.append(j); bs.append(b); ws.append(w)
+                                ps.append(generate.shard_ptr(slabs[j][it], w, job.blocks[b].job_offset))
+                        svc.round(np.array(js, np.int32), np.array(bs, np.int32), np.array(ws, np.int32),
+                                  np.array(ps, np.uint64), ready, B.PS_ROUND_INPUTS_COMPLETE, stream)
+                    if it == 1:
+                        svc.join(stream)            # one agent joining flushes what the others have queued: allowed
+                svc.join(stream)
+                stream.synchronize()
+            except Exception as e:      # noqa: BLE001
+                errors.append((j, e))
+
+        threads = [threading.Thread(target=agent, args=(j,)) for j in range(len(jobs))]
+        [t.start() for t in threads]
+        [t.join() for t in threads]
+        assert not errors, errors
+        for it in range(iters):
+            for j, job in enumerate(cfg.jobs):
+                host = to_np(slabs[j][it])
+                ready = []
+                for b in job.blocks:
+                    for w in range(job.num_workers):
+                        pair.ora.push(j, b.block, w, host[w, b.job_offset:b.job_offset + b.nelem])
+                    ready.append((j, b.block))
+                pair.ora.aggregate(ready)
+        assert pair.compare(iters) == cfg.num_params
+    finally:
+        pair.close()
