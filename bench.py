@@ -46,7 +46,7 @@ _SHARED_SOURCES = ("ps_types.cuh", "ps_math.cuh", "ps_rows.cuh")
 NCU_TRAFFIC = {
     "ps_aggregate_ldg_kernel": {"sources": _SHARED_SOURCES + ("ps_kernel_ldg.cuh",), "kernel_sha": "4733ace9e33e",
                                 "dram_bytes_per_algorithmic_byte": 0.980},
-    "ps_aggregate_bulk_kernel": {"sources": _SHARED_SOURCES + ("ps_kernel_bulk.cuh",), "kernel_sha": "504eed6eb701",
+    "ps_aggregate_bulk_kernel": {"sources": _SHARED_SOURCES + ("ps_kernel_bulk.cuh",), "kernel_sha": "5610a06cdf42",
                                  "dram_bytes_per_algorithmic_byte": 0.984},
 }
 

@@ -13,10 +13,10 @@
 // the direct-load kernel — and on the last stage apply the optimizer and store
 // parameters and state with 128-bit stores.  The ring keeps 192 KB per SM in
 // flight whatever W is.  A tenth warp collects each finished chunk's partial
-// sums of squares and draws the tickets that count a task's chunks when the
-// CTA has run out of work: done by the producer, per chunk, those round trips
-// to memory and their fences were the kernel's bottleneck — the producer has
-// about a thousand cycles per stage to keep the ring full.
+// sums of squares and draws the tickets that count a task's chunks once per
+// eight chunks: done by the producer, per chunk, those round trips to memory
+// and their fences were the kernel's bottleneck — the producer has about a
+// thousand cycles per stage to keep the ring full.
 //
 // Chunks that cannot use bulk copies (a shard pointer that is not 16-byte
 // aligned, fewer elements than one vector) are handed to the consumers as
