@@ -137,6 +137,32 @@ def test_recycling_moves_a_light_aggregator_onto_others():
     assert o.remove_job(a) == 1 and o.num_alive() == 1
 
 
+def test_best_fit_prefers_a_tighter_aggregator_with_a_higher_index():
+    # n0 holds 4 + 3 (3 free), n1 holds 7.5 (2.5 free): a task of 2 fits both and goes to n1,
+    # the one with the fewest free slots — not to the first that fits
+    o = O.AssignmentOracle()
+    a, x, b = o.add_job(10), o.add_job(10), o.add_job(10)
+    assert [o.assign(a, 4)[1], o.assign(a, 3)[1], o.assign(x, 7.5)[1]] == [0, 0, 1]
+    assert o.estimate(0, b, 2) == (3.0, 2) and o.estimate(1, b, 2) == (2.5, 2)
+    assert o.assign(b, 2)[1] == 1
+
+
+def test_recycling_empties_the_least_loaded_aggregator_and_leaves_the_heavy_one_alone():
+    # Section 3.3.2: after job x has left, n1 holds one task of 2 and n0 holds 4 + 3.  Either could
+    # be emptied onto the other (7 fits into n1's 8 free slots, 2 into n0's 3); it is the lightly
+    # loaded one that is recycled: one task moves, the heavy Aggregator's tasks stay where they are.
+    o = O.AssignmentOracle()
+    a, x, b = o.add_job(10), o.add_job(10), o.add_job(10)
+    ta, tb = o.assign(a, 4)[0], o.assign(a, 3)[0]
+    o.assign(x, 7.5)
+    tc, n = o.assign(b, 2)
+    assert n == 1 and o.num_alive() == 2
+    assert o.remove_job(x) == 1 and o.num_alive() == 1
+    assert o.N[0].alive and not o.N[1].alive
+    assert o.where[ta] == o.where[tb] == o.where[tc] == 0
+    assert o.load(0) == 9
+
+
 def test_outlier_rule():
     # cycle 12, 7 units gone, 3 units of scheduled work still to run: 2 units are spare
     assert O.outlier_fits(12, 7, 3, 2)
@@ -183,6 +209,20 @@ def test_planner_reproduces_the_papers_toy_numbers(_lib):
     assert n1 == 0 and ji["current"] == g["B.duration_after"]
     assert round(100 * ji["loss"]) == g["B.loss_percent_rounded"]
     assert B.Planner.outlier_fits(12, 7, 3, 2) and not B.Planner.outlier_fits(12, 7, 3, 2.5)
+
+
+def test_planner_best_fit_and_recycling_of_the_lightest_as_the_oracle(_lib):
+    # the two hand-worked cases of the oracle's pins, through the library's planner
+    p = B.Planner(0.1)
+    a, x, b = p.add_job(10), p.add_job(10), p.add_job(10)
+    ta, tb = p.assign(a, 4), p.assign(a, 3)
+    assert (ta[1], tb[1], p.assign(x, 7.5)[1]) == (0, 0, 1)
+    tc = p.assign(b, 2)
+    assert tc[1] == 1                                   # 2.5 free beats 3 free: best fit, not first fit
+    assert p.remove_job(x) == 1 and p.num_aggregators() == (2, 1)
+    assert p.aggregator_info(0)["alive"] and not p.aggregator_info(1)["alive"]
+    assert [p.task_info(t)[1] for t in (ta[0], tb[0], tc[0])] == [0, 0, 0]      # only the light Aggregator's task moved
+    assert p.aggregator_info(0)["load"] == 9
 
 
 @pytest.mark.parametrize("seed", [0, 1, 2, 3])

@@ -123,3 +123,64 @@ def test_every_planted_mistake_fails_a_pin(tmp_path):
         survived = [n for n, ok in zip(names, pool.map(lambda n: _pins_pass(_build(tmp, n, MUTANTS[n])), names)) if ok]
     assert not survived, "no pin notices: " + "; ".join(survived)
     assert len(names) >= 30
+
+
+# ---------------------------------------------------------------- the assignment oracle (Pseudocode 1)
+
+ASSIGN_SRC = os.path.join(ROOT, "oracle", "assignment.py")
+ASSIGN_MUTANTS = {
+    "cycle: the shortest period instead of the longest": [
+        ("return max((self.D[j] for j in js), default=0.0)", "return min((self.D[j] for j in js), default=0.0)")],
+    "stretched duration: one slot too many": [("max(D_j, C / r)", "max(D_j, C / (r + 1))")],
+    "loss relative to the profiled duration": [("return (d_j - D_j) / d_j", "return (d_j - D_j) / D_j")],
+    "loss limit doubled": [(">= self.loss_limit", ">= 2 * self.loss_limit")],
+    "estimated cycle ignores the new job": [("C_est = max(self.cycle(n), self.D[k])", "C_est = max(self.cycle(n), 0.0)")],
+    "free slots: multiplicity dropped": [
+        ("free -= floor_ratio(C_est, d_j) * sum(self.N[n].tasks.get(j, {}).values())",
+         "free -= sum(self.N[n].tasks.get(j, {}).values())")],
+    "needed slots: multiplicity dropped": [
+        ("need = floor_ratio(C_est, stretched_duration(self.D[k], C_est)) * e_t", "need = e_t")],
+    "worst fit": [("F < best[1]", "F > best[1]")],
+    "first fit": [("(best is None or F < best[1])", "best is None")],
+    "any Aggregator with a free slot fits": [("F >= need - 1e-12", "F > 0")],
+    "the new task's own job is not examined": [("sorted(set(self.N[n].jobs()) | {k})", "sorted(set(self.N[n].jobs()))")],
+    "recycling starts from the heaviest": [("n = min(live, key=lambda i: (self.load(i), i))", "n = max(live, key=lambda i: (self.load(i), i))")],
+    "recycling may re-place onto the same Aggregator": [("allow_new=False, exclude=n", "allow_new=False, exclude=-1")],
+    "outlier: scheduled requests not reserved": [
+        ("return (C_n - now_in_cycle) - remaining_scheduled >= e_late - 1e-12", "return (C_n - now_in_cycle) >= e_late - 1e-12")],
+    "floor without its guard": [("int(math.floor(a / b * (1.0 + 1e-9) + 1e-12))", "int(math.floor(a / b))")],
+    "load: multiplicity dropped": [("tot += floor_ratio(C, d) * sum(self.N[n].tasks[j].values())", "tot += sum(self.N[n].tasks[j].values())")],
+    "empty Aggregators are not released": [("            if a.alive and not a.jobs():\n                a.alive = False\n                released += 1",
+                                            "            if False:\n                a.alive = False\n                released += 1")],
+}
+
+
+def _assignment_pins_pass(tmp, name, edits):
+    src = open(ASSIGN_SRC).read()
+    for old, new in edits:
+        assert src.count(old) >= 1, "mutant %r: text %r not in the assignment oracle" % (name, old)
+        src = src.replace(old, new)
+    path = os.path.join(tmp, "assignment_" + "".join(c if c.isalnum() else "_" for c in name) + ".py")
+    open(path, "w").write(src)
+    # the child loads the changed file as oracle.assignment, then runs the oracle's own pins
+    # (the planner-parity tests need the library and are not what is being examined here)
+    code = ("import sys, importlib.util; sys.path.insert(0, %r); import oracle; "
+            "spec = importlib.util.spec_from_file_location('oracle.assignment', %r); m = importlib.util.module_from_spec(spec); "
+            "sys.modules['oracle.assignment'] = m; spec.loader.exec_module(m); oracle.assignment = m; "
+            "import pytest; sys.exit(pytest.main(['-x', '-q', '-p', 'no:cacheprovider', '-k', 'not planner', 'tests/test_assignment.py']))"
+            % (ROOT, path))
+    try:
+        r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, capture_output=True, text=True, timeout=120)
+    except subprocess.TimeoutExpired:
+        return False                     # a mistake that never terminates is noticed too
+    assert r.returncode in (0, 1), "the pin run itself broke:\n" + r.stdout[-2000:] + r.stderr[-2000:]
+    return r.returncode == 0
+
+
+def test_every_mistake_planted_in_the_assignment_oracle_fails_a_pin(tmp_path):
+    tmp = str(tmp_path)
+    assert _assignment_pins_pass(tmp, "control", []), "the unchanged assignment oracle must pass its pins"
+    names = list(ASSIGN_MUTANTS)
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        survived = [n for n, ok in zip(names, pool.map(lambda n: _assignment_pins_pass(tmp, n, ASSIGN_MUTANTS[n]), names)) if ok]
+    assert not survived, "no pin notices: " + "; ".join(survived)
