@@ -184,3 +184,53 @@ def test_every_mistake_planted_in_the_assignment_oracle_fails_a_pin(tmp_path):
     with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
         survived = [n for n, ok in zip(names, pool.map(lambda n: _assignment_pins_pass(tmp, n, ASSIGN_MUTANTS[n]), names)) if ok]
     assert not survived, "no pin notices: " + "; ".join(survived)
+
+
+# ---------------------------------------------------------------- the oracle's service semantics (Python)
+
+SERVICE_SRC = os.path.join(ROOT, "oracle", "aggregator.py")
+SERVICE_PINS = ["tests/test_oracle_pins.py", "tests/test_oracle_service_pins.py", "tests/test_rows.py"]
+SERVICE_MUTANTS = {
+    "step counter does not advance": [("            b.step += 1\n", "            b.step += 0\n")],
+    "shards summed in arrival order, not worker order": [
+        ("[b.pushed[w] for w in range(hp.num_workers)]", "list(b.pushed.values())")],
+    "pushes not cleared by an aggregate": [("                b.pushed = {}\n", "                pass\n")],
+    "a worker may push twice": [("        if worker in b.pushed:\n            raise ValueError(\"duplicate push\")", "        if False:\n            raise ValueError(\"duplicate push\")")],
+    "a task that is not ready is skipped, not refused": [("                raise RuntimeError(\"not ready\")", "                continue")],
+    "a task may be listed twice": [("            if key in seen:\n                raise ValueError(\"task listed twice\")", "            if False:\n                raise ValueError(\"task listed twice\")")],
+    "unlisted rows are -0.0": [("        dense = np.zeros((b.nelem // row_len, row_len), dtype=_grad_np_dtype(hp))",
+                                "        dense = -np.zeros((b.nelem // row_len, row_len), dtype=_grad_np_dtype(hp)) if _grad_np_dtype(hp) == np.float32 else np.zeros((b.nelem // row_len, row_len), dtype=np.uint16)")],
+    "row ids may repeat": [("np.any(np.diff(ids) <= 0)", "np.any(np.diff(ids) < 0)")],
+    "migration forgets the context": [("        b.ctx = dst_ctx\n", "        pass\n")],
+    "migration restarts the step counter": [("        b.ctx = dst_ctx\n", "        b.ctx = dst_ctx\n        b.step = 0\n")],
+    "migration drops the optimizer state": [("        b.p, b.s0 = b.p.copy(), b.s0.copy()", "        b.p, b.s0 = b.p.copy(), np.zeros_like(b.s0)")],
+    "state does not start at zero": [("        s0 = np.zeros(nelem, np.float32)\n", "        s0 = np.ones(nelem, np.float32)\n")],
+    "norms accumulate over iterations": [("                b.sqnorm = s\n", "                b.sqnorm += s\n")],
+}
+
+
+def _service_pins_pass(tmp, name, edits):
+    src = open(SERVICE_SRC).read()
+    for old, new in edits:
+        assert src.count(old) >= 1, "mutant %r: text %r not in the oracle's service code" % (name, old)
+        src = src.replace(old, new)
+    path = os.path.join(tmp, "aggregator_" + "".join(c if c.isalnum() else "_" for c in name) + ".py")
+    open(path, "w").write(src)
+    code = ("import sys, importlib.util; sys.path.insert(0, %r); import oracle; "
+            "spec = importlib.util.spec_from_file_location('oracle.aggregator', %r); m = importlib.util.module_from_spec(spec); "
+            "sys.modules['oracle.aggregator'] = m; spec.loader.exec_module(m); oracle.aggregator = m; "
+            "import pytest; sys.exit(pytest.main(['-x', '-q', '-p', 'no:cacheprovider', '-m', 'not gpu'] + %r))"
+            % (ROOT, path, SERVICE_PINS))
+    r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, capture_output=True, text=True, timeout=300,
+                       env=dict(os.environ, OMP_NUM_THREADS="2"))
+    assert r.returncode in (0, 1), "the pin run itself broke:\n" + r.stdout[-2000:] + r.stderr[-2000:]
+    return r.returncode == 0
+
+
+def test_every_mistake_planted_in_the_oracles_service_semantics_fails_a_pin(tmp_path):
+    tmp = str(tmp_path)
+    assert _service_pins_pass(tmp, "control", []), "the unchanged oracle must pass its pins"
+    names = list(SERVICE_MUTANTS)
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        survived = [n for n, ok in zip(names, pool.map(lambda n: _service_pins_pass(tmp, n, SERVICE_MUTANTS[n]), names)) if ok]
+    assert not survived, "no pin notices: " + "; ".join(survived)

@@ -184,6 +184,34 @@ def test_fp32_special_values_travel_like_ieee_binary32(opt, kernel, shift):
         pair.close()
 
 
+@pytest.mark.parametrize("kernel", [1, 2, 3], ids=["ldg", "bulk", "inline"])
+@pytest.mark.parametrize("dt", [configs.F32, configs.BF16])
+def test_the_sum_follows_worker_order_not_arrival_order(kernel, dt):
+    """g0 = 2^24, g1 = g2 = 1 (all exact in bf16 too): in worker order the ones are rounded
+    away one at a time and G = 2^24; summed as they ARRIVE (2, 1, 0) G would be 2^24 + 2."""
+    n = 12289
+    cfg = tiny_config([n], 3, grad_dtype=dt, lr=1.0, momentum=0.0, weight_decay=0.0)
+    pair = Pair(cfg, kernel=kernel)
+    try:
+        vals = {0: 2.0 ** 24, 1: 1.0, 2: 1.0}
+        keep = []
+        for w in (2, 1, 0):
+            t = torch.full((n,), vals[w], dtype=torch.float32, device="cuda")
+            host = np.full(n, vals[w], np.float32)
+            if dt == configs.BF16:
+                t = t.to(torch.bfloat16)
+                host = (host.view(np.uint32) >> 16).astype(np.uint16)
+            keep.append(t)
+            pair.svc.push(0, 0, w, t)
+            pair.ora.push(0, 0, w, host)
+        pair.aggregate([(0, 0)])
+        p, v, _, _ = pair.gpu_block(0, 0)
+        assert np.array_equal(v, pair.ora.state(0, 0)[0]) and np.array_equal(p, pair.ora.pull(0, 0))
+        assert float(v[0]) == float(v[-1]) == 2.0 ** 24
+    finally:
+        pair.close()
+
+
 def test_small_rounds_travel_as_kernel_parameters_and_slots_stay_clean():
     """A round whose table fits the kernel-parameter limit launches without an
     upload.  Tasks of several chunks count their chunks in per-slot device
