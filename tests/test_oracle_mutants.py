@@ -18,7 +18,7 @@ import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 SRC = os.path.join(ROOT, "oracle", "ps_oracle.cpp")
-PINS = ["tests/test_oracle_pins.py", "tests/test_oracle_ieee.py"]
+PINS = ["tests/test_oracle_pins.py", "tests/test_oracle_ieee.py", "tests/test_oracle_service_pins.py"]
 
 # name -> [(text in the oracle's source, replacement), ...]; every text must occur
 MUTANTS = {
@@ -87,6 +87,12 @@ MUTANTS = {
     "norm: not squared": [("sq += (double)G * (double)G;", "sq += (double)G;"), ("sq += G * G;", "sq += G;")],
     "norm: taken before the scale": [("    G = G * gs;\n    sq += (double)G * (double)G;", "    sq += (double)G * (double)G;\n    G = G * gs;"),
                                      ("    G = G * gs;\n    sq += G * G;", "    sq += G * G;\n    G = G * gs;")],
+    "blocks: the last task of a batch is skipped": [
+        ("for (int b = 0; b < n; ++b) bad |= (oracle_block_step_f32(&tasks[b]) != 0);",
+         "for (int b = 0; b < n - 1; ++b) bad |= (oracle_block_step_f32(&tasks[b]) != 0);")],
+    "elements: the last element of a block is skipped": [("for (uint64_t i = 0; i < k->nelem; ++i) {", "for (uint64_t i = 0; i + 1 < k->nelem; ++i) {")],
+    "bf16 array widening stops one short": [("for (uint64_t i = 0; i < n; ++i) out[i] = oracle_bf16_to_f32(bits[i]);",
+                                             "for (uint64_t i = 0; i + 1 < n; ++i) out[i] = oracle_bf16_to_f32(bits[i]);")],
     "bf16: shifted by 15": [("(uint32_t)bits << 16", "(uint32_t)bits << 15")],
     "bf16: low half of the word": [("(uint32_t)bits << 16", "(uint32_t)bits")],
 }

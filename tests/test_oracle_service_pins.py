@@ -114,3 +114,10 @@ def test_migration_moves_the_block_to_the_named_context_with_everything_it_holds
     assert list(o.state(0, 0)[0]) == [1.5, 3.0] and o.block_stats(0, 0)[1] == 2
     with pytest.raises(ValueError):
         o.migrate_block(0, 0, 3)
+
+
+def test_array_widening_of_bf16_covers_every_element():
+    # 0x3F80 = 1.0, 0x4000 = 2.0, 0xC040 = -3.0, 0x0001 = 2^-133 (a bf16 subnormal): the last one too
+    got = A.widen_bf16(np.array([0x3F80, 0x4000, 0xC040, 0x0001], np.uint16))
+    assert bits(got) == [0x3F800000, 0x40000000, 0xC0400000, 0x00010000]
+    assert A.widen_bf16(np.array([0xC040], np.uint16)).tolist() == [-3.0]
