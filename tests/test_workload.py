@@ -73,6 +73,13 @@ def test_generators_are_deterministic_and_shaped():
     assert g0.shape == (4, 1 << 20) and abs(g0.std().item() - 1e-2) < 1e-4
     p = generate.init_params(cfg, 0)
     assert abs(p.std().item() - 0.05) < 1e-3
+    # every worker draws its own gradients (identical shards would hide a wrong worker order or a
+    # dropped worker from every parity test), and they are uncorrelated
+    for a in range(4):
+        for b in range(a + 1, 4):
+            assert not torch.equal(g0[a], g0[b])
+            assert abs(float((g0[a] * g0[b]).mean()) / 1e-4) < 0.01
+    assert abs(g0.mean().item()) < 1e-4 and (g0 != 0).float().mean() > 0.999
 
 
 def test_row_sparse_embedding_and_bf16_rounding():
